@@ -1,0 +1,182 @@
+/*
+ * scar.h - C ABI of the SCAR checkpoint-and-recover parameter pass on one GPU.
+ *
+ * The library keeps a running checkpoint z of a caller-owned parameter buffer
+ * x in device memory and offers the two strategies of the paper's Section 4:
+ *   - prioritized partial checkpoints (Section 4.2, protocol of Section 4.3):
+ *     score every block by its distance to the saved copy, take the fraction
+ *     r with the largest scores, refresh z on those blocks and emit them as a
+ *     contiguous payload;
+ *   - partial recovery (Section 4.1): restore only the lost blocks from z and
+ *     report the perturbation ||z_S - x_S|| that the iteration-cost bound of
+ *     Theorem 3.2 depends on.
+ *
+ * Terms.  An element is 4 bytes (float32 or int32).  A block is a contiguous
+ * element range and is the unit of scoring, selection and loss (the paper's
+ * "parameter": a row, a layer or a shard of a layer, Section 5.1).  A shard is
+ * a contiguous range of blocks standing for one parameter-server node.
+ *
+ * Conventions for every call.
+ *   - Return value: SCAR_OK (0) or a negative SCAR_ERR_* code; nothing throws.
+ *     Arguments are validated before any GPU work is enqueued, so a call that
+ *     fails validation leaves every buffer untouched.
+ *   - Pointer names say where the memory lives: d_* device, h_* host.
+ *   - All GPU work of a context runs on the CUDA stream given at init, in call
+ *     order.  A call whose result pointer `out` is NULL only enqueues; with a
+ *     non-NULL `out` it also waits for the stream and fills `out`.
+ *   - One context serves one caller at a time (no internal locking).
+ *   - There is no CPU fallback: without a usable CUDA device init fails.
+ */
+#ifndef SCAR_H
+#define SCAR_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct scar_ctx scar_ctx; /* opaque; created by scar_ckpt_init, freed by scar_ckpt_destroy */
+
+/* Element type.  SCAR_F32 scores blocks by the squared l2 distance (the norm of
+ * the appendix proofs of Theorems 4.1/4.2); SCAR_I32 by the integer l1 distance
+ * (twice the length-scaled total variation that Appendix C uses for LDA). */
+typedef enum { SCAR_F32 = 0, SCAR_I32 = 1 } scar_dtype;
+
+enum {
+    SCAR_OK = 0,
+    SCAR_ERR_INVALID_ARG = -1, /* NULL where not allowed, r outside [0,1], k > B, misaligned x ... */
+    SCAR_ERR_LAYOUT = -2,      /* inconsistent block geometry */
+    SCAR_ERR_ALLOC = -3,       /* device or host allocation failed */
+    SCAR_ERR_CUDA = -4,        /* a CUDA runtime call or kernel launch failed */
+    SCAR_ERR_STATE = -5,       /* call not valid in the context's current state */
+    SCAR_ERR_TIMEOUT = -6      /* reserved: a bounded device-side wait gave up */
+};
+
+/* Block geometry of the flat buffer of n_elems elements.
+ *   Implicit form (block_offsets == NULL): rows of row_elems elements
+ *   (0 = one row of n_elems; otherwise n_elems % row_elems == 0), each cut into
+ *   blocks of block_elems; the last block of a row may be shorter; blocks never
+ *   cross a row end.  n_blocks is ignored.
+ *   Explicit form: block_offsets is a HOST array of n_blocks + 1 non-decreasing
+ *   element offsets with block_offsets[0] == 0 and block_offsets[n_blocks] ==
+ *   n_elems; it is copied during init.  row_elems / block_elems are ignored.
+ * n_shards >= 1; shard s owns blocks [floor(s*B/S), floor((s+1)*B/S)).
+ * At most 2^32 - 1 blocks. */
+typedef struct {
+    uint64_t n_elems;
+    uint64_t row_elems;
+    uint32_t block_elems;
+    uint32_t n_shards;
+    const uint64_t *block_offsets;
+    uint64_t n_blocks;
+} scar_layout;
+
+typedef struct {
+    uint64_t k;                /* blocks saved */
+    uint64_t payload_elems;    /* elements in the payload = poff[k] */
+    uint64_t nonfinite_blocks; /* SCAR_F32: blocks whose score was NaN or +Inf (ranked first) */
+} scar_save_info;
+
+typedef struct {
+    double l2;            /* SCAR_F32: ||z_S - x_S||_2 ; 0 for SCAR_I32 */
+    uint64_t l1;          /* SCAR_I32: sum_{i in S} |z_i - x_i| ; 0 for SCAR_F32 */
+    uint64_t lost_blocks; /* |S| in blocks */
+    uint64_t lost_elems;  /* |S| in elements */
+} scar_norm_info;
+
+/* Creates a context over the caller's device buffer d_x (n_elems elements of
+ * type dt, 16-byte aligned, owned by the caller, must stay valid and in place
+ * until destroy) and initialises the running checkpoint z := x (Section 4.2:
+ * the running checkpoint starts from the initial parameter values).  Allocates
+ * z, the score/selection arrays and a payload buffer of n_elems elements on the
+ * current CUDA device.  cuda_stream is a cudaStream_t (NULL = default stream).
+ * Waits for the stream before returning.  On error *out is NULL. */
+int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *layout, void *cuda_stream);
+
+/* Checkpoint step 1 of Section 4.3 alone: recomputes score_b = dist(x_b, z_b)
+ * for every block into the context's score array (float32 squared l2, or
+ * uint64 l1).  Enqueue only. */
+int scar_ckpt_block_scores(scar_ctx *ctx);
+
+/* One prioritized partial checkpoint (Section 4.2; steps 1, 3, 4 of the
+ * checkpoint protocol in Section 4.3): scores all blocks, selects the
+ * k = round(r*B) highest (halves away from zero; at least 1 if r > 0; ties to
+ * the lowest block id; NaN/Inf scores rank first), writes their ids ascending to
+ * sel[k], their payload offsets to poff[k+1], copies x over them into the
+ * payload in that order and refreshes z_b := x_b on them.  r = 1 is the
+ * traditional full checkpoint.  r outside [0,1] or NaN: SCAR_ERR_INVALID_ARG. */
+int scar_ckpt_priority_save(scar_ctx *ctx, double r, scar_save_info *out);
+
+/* Same with the block count given directly (0 <= k <= B). */
+int scar_ckpt_priority_save_k(scar_ctx *ctx, uint64_t k, scar_save_info *out);
+
+/* Partial recovery (Section 4.1; recovery step 2 of Section 4.3): for every
+ * block of every lost shard, accumulates the perturbation of the appendix proof
+ * of Theorem 4.1, ||z_S - x_S||, from the values x still holds, then overwrites
+ * x_b := z_b.  Blocks outside S and all of z are left untouched.
+ * h_lost_shards: HOST array of n_shards bytes, 0 = alive, non-zero = lost. */
+int scar_recover_partial(scar_ctx *ctx, const uint8_t *h_lost_shards, scar_norm_info *out);
+
+/* Same with an arbitrary lost set: d_lost_blocks is a DEVICE array of B bytes
+ * (0 alive, non-zero lost), read when the enqueued work runs. */
+int scar_recover_partial_blocks(scar_ctx *ctx, const uint8_t *d_lost_blocks, scar_norm_info *out);
+
+/* The perturbation a recovery of the given lost set would cause, without
+ * writing anything.  NULL mask = every block lost = full recovery, whose
+ * perturbation is x^(T) - x^(C) (Example 2.3). */
+int scar_perturbation_norm(scar_ctx *ctx, const uint8_t *h_lost_shards, scar_norm_info *out);
+int scar_perturbation_norm_blocks(scar_ctx *ctx, const uint8_t *d_lost_blocks, scar_norm_info *out);
+
+/* Host-buffer forms for callers whose parameters live in host memory.
+ * save_host: copies n_elems elements from h_x into the context's x, runs the
+ * save, then copies back payload_elems elements to h_payload (capacity n_elems
+ * elements), k ids to h_sel (capacity k) and k+1 offsets to h_poff.  Always
+ * waits for completion; `out` must not be NULL.
+ * recover_host: copies the lost shards' element ranges of h_x (the values the
+ * failed nodes last held) into x, runs the recovery, and copies the recovered
+ * ranges back into h_x; other ranges of h_x are neither read nor written. */
+int scar_ckpt_priority_save_host(scar_ctx *ctx, const void *h_x, double r, void *h_payload, uint32_t *h_sel,
+                                 uint64_t *h_poff, scar_save_info *out);
+int scar_recover_partial_host(scar_ctx *ctx, void *h_x, const uint8_t *h_lost_shards, scar_norm_info *out);
+
+/* Replaces the running checkpoint by n_elems elements read from the device
+ * buffer d_z_src (e.g. a checkpoint read back from storage).  Enqueue only. */
+int scar_ckpt_load(scar_ctx *ctx, const void *d_z_src);
+
+/* Waits for the stream and returns the results of the most recent save and the
+ * most recent recover/norm call (either pointer may be NULL). */
+int scar_ckpt_last_info(scar_ctx *ctx, scar_save_info *save, scar_norm_info *norm);
+
+/* Borrowed device pointers (any may be NULL to skip): z (n_elems elements),
+ * scores (B float32 for SCAR_F32, B uint64 for SCAR_I32; as of the last
+ * scoring), sel (k uint32), poff (k+1 uint64), payload.  Valid until destroy;
+ * contents change with the next save. */
+int scar_ckpt_view(scar_ctx *ctx, const void **d_z, const void **d_scores, const uint32_t **d_sel,
+                   const uint64_t **d_poff, const void **d_payload);
+
+/* Geometry as the library resolved it. */
+uint64_t scar_ckpt_n_blocks(const scar_ctx *ctx);
+
+/* Kernels this context has launched so far (its own kernels only). */
+uint64_t scar_ckpt_launch_count(const scar_ctx *ctx);
+
+/* Optional per-phase device timing.  With enable != 0 every later call brackets
+ * its phases with CUDA events on the context's stream.  phase_ms receives the
+ * duration of the most recent call's phases, in milliseconds, after waiting for
+ * the stream: [0] block scores, [1] selection, [2] pack + cache refresh,
+ * [3] restore / norm pass, [4] final reduction; phases a call did not run
+ * read 0. */
+int scar_ckpt_profile(scar_ctx *ctx, int enable);
+int scar_ckpt_profile_read(scar_ctx *ctx, float phase_ms[5]);
+
+/* Waits for the stream, frees everything the context owns (never x). */
+int scar_ckpt_destroy(scar_ctx *ctx);
+
+/* Static description of an error code. */
+const char *scar_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SCAR_H */

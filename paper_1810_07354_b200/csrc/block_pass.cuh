@@ -1,0 +1,280 @@
+// Streaming pass over the two parameter streams x (live) and z (running
+// checkpoint), block by block: per-block distance for the checkpoint scores
+// (Section 4.3, checkpoint step 1) and, for recovery, the same sum over the lost
+// blocks fused with x_b := z_b (Section 4.1; appendix proof of Theorem 4.1).
+//
+// A group of G consecutive lanes (G = 4..32, a power of two) owns one block at
+// a time.  Each lane issues 16-byte loads G vectors apart, four per stream in
+// flight, and keeps four independent accumulators; the group total is formed
+// with xor-shuffles, so the summation order depends only on G and the block
+// length, never on scheduling: results are bit-reproducible run to run.
+#pragma once
+#include <type_traits>
+
+#include "geom.cuh"
+
+namespace scar {
+
+constexpr int kThreads = 256;
+
+template <typename T> struct Elem;
+
+// float32 elements: squared l2 distance.  Inner chains are fp32 (at most 64
+// vectors per accumulator between flushes), the outer sum and the cross-lane
+// reduction are fp64, so long blocks do not lose accuracy.
+template <> struct Elem<float> {
+    using vec_t = float4;
+    using wide_t = double;   // what a group reduces to
+    using score_t = float;   // what is stored per block
+    using acc_t = float;
+    static __device__ __forceinline__ void add(acc_t &a, float x, float z) {
+        float d = x - z;
+        a = fmaf(d, d, a);
+    }
+    static __device__ __forceinline__ void add4(acc_t &a, const vec_t &x, const vec_t &z) {
+        add(a, x.x, z.x); add(a, x.y, z.y); add(a, x.z, z.z); add(a, x.w, z.w);
+    }
+    static constexpr bool kFlush = true;
+};
+
+// int32 elements: integer l1 distance, exact in 64 bits (|x - z| < 2^32).
+template <> struct Elem<int> {
+    using vec_t = int4;
+    using wide_t = unsigned long long;
+    using score_t = unsigned long long;
+    using acc_t = unsigned long long;
+    static __device__ __forceinline__ void add(acc_t &a, int x, int z) {
+        unsigned d = x > z ? (unsigned)x - (unsigned)z : (unsigned)z - (unsigned)x;
+        a += d;
+    }
+    static __device__ __forceinline__ void add4(acc_t &a, const vec_t &x, const vec_t &z) {
+        add(a, x.x, z.x); add(a, x.y, z.y); add(a, x.z, z.z); add(a, x.w, z.w);
+    }
+    static constexpr bool kFlush = false;
+};
+
+template <typename V> __device__ __forceinline__ V ld_stream(const V *p) { return __ldcs(p); }
+template <typename V> __device__ __forceinline__ void st_stream(V *p, const V &v) { __stcs(p, v); }
+
+template <int G, typename W> __device__ __forceinline__ W group_sum(W v) {
+#pragma unroll
+    for (int o = G / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Distance sum of one block over the lanes of a group; every lane returns the
+// group total.  len == 0 is allowed (the lane then only takes part in the
+// shuffles).  WRITE: also store z over x.  VEC: block starts/ends are 16-byte
+// aligned, so the whole block moves as 16-byte vectors; otherwise element-wise.
+template <typename T, int G, bool VEC, bool WRITE>
+__device__ __forceinline__ typename Elem<T>::wide_t block_distance(T *__restrict__ x, const T *__restrict__ z,
+                                                                   uint64_t beg, uint64_t len, int lane) {
+    using E = Elem<T>;
+    using vec_t = typename E::vec_t;
+    using acc_t = typename E::acc_t;
+    using wide_t = typename E::wide_t;
+    acc_t a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+    wide_t total = 0;
+    if (VEC) {
+        vec_t *xv = reinterpret_cast<vec_t *>(x + beg);
+        const vec_t *zv = reinterpret_cast<const vec_t *>(z + beg);
+        const uint64_t nvec = len >> 2;
+        uint64_t v = lane;
+        unsigned it = 0;
+        for (; v + 3 * G < nvec; v += 4 * G) {
+            vec_t x0 = ld_stream(xv + v), x1 = ld_stream(xv + v + G);
+            vec_t x2 = ld_stream(xv + v + 2 * G), x3 = ld_stream(xv + v + 3 * G);
+            vec_t z0 = ld_stream(zv + v), z1 = ld_stream(zv + v + G);
+            vec_t z2 = ld_stream(zv + v + 2 * G), z3 = ld_stream(zv + v + 3 * G);
+            E::add4(a0, x0, z0); E::add4(a1, x1, z1); E::add4(a2, x2, z2); E::add4(a3, x3, z3);
+            if (WRITE) {
+                st_stream(xv + v, z0); st_stream(xv + v + G, z1);
+                st_stream(xv + v + 2 * G, z2); st_stream(xv + v + 3 * G, z3);
+            }
+            if (E::kFlush && (++it & 63u) == 0) {
+                total += ((wide_t)a0 + (wide_t)a1) + ((wide_t)a2 + (wide_t)a3);
+                a0 = a1 = a2 = a3 = 0;
+            }
+        }
+        for (; v < nvec; v += G) {
+            vec_t x0 = ld_stream(xv + v);
+            vec_t z0 = ld_stream(zv + v);
+            E::add4(a0, x0, z0);
+            if (WRITE) st_stream(xv + v, z0);
+        }
+    } else {
+        T *xs = x + beg;
+        const T *zs = z + beg;
+        uint64_t i = lane;
+        unsigned it = 0;
+        for (; i + 3 * G < len; i += 4 * G) {
+            T x0 = ld_stream(xs + i), x1 = ld_stream(xs + i + G), x2 = ld_stream(xs + i + 2 * G),
+              x3 = ld_stream(xs + i + 3 * G);
+            T z0 = ld_stream(zs + i), z1 = ld_stream(zs + i + G), z2 = ld_stream(zs + i + 2 * G),
+              z3 = ld_stream(zs + i + 3 * G);
+            E::add(a0, x0, z0); E::add(a1, x1, z1); E::add(a2, x2, z2); E::add(a3, x3, z3);
+            if (WRITE) {
+                st_stream(xs + i, z0); st_stream(xs + i + G, z1);
+                st_stream(xs + i + 2 * G, z2); st_stream(xs + i + 3 * G, z3);
+            }
+            if (E::kFlush && (++it & 255u) == 0) {
+                total += ((wide_t)a0 + (wide_t)a1) + ((wide_t)a2 + (wide_t)a3);
+                a0 = a1 = a2 = a3 = 0;
+            }
+        }
+        for (; i < len; i += G) {
+            T x0 = ld_stream(xs + i);
+            T z0 = ld_stream(zs + i);
+            E::add(a0, x0, z0);
+            if (WRITE) st_stream(xs + i, z0);
+        }
+    }
+    total += ((wide_t)a0 + (wide_t)a1) + ((wide_t)a2 + (wide_t)a3);
+    return group_sum<G, wide_t>(total);
+}
+
+// ---- a1: score of every block ----------------------------------------------
+
+struct SelState;  // select.cuh
+
+template <typename T, int G, bool VEC>
+__global__ void __launch_bounds__(kThreads)
+k_block_scores(const T *__restrict__ x, const T *__restrict__ z, Geom g, typename Elem<T>::score_t *__restrict__ score,
+               unsigned long long *key_or, unsigned *hist0, int hist0_len) {
+    using E = Elem<T>;
+    const int lane = threadIdx.x & (G - 1);
+    const uint64_t grp = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
+    const bool valid = grp < g.n_blocks;
+    uint64_t beg = 0, len = 0;
+    if (valid) g.range((uint32_t)grp, beg, len);
+    typename E::wide_t s = block_distance<T, G, VEC, false>(const_cast<T *>(x), z, beg, len, lane);
+    if (valid && lane == 0) {
+        typename E::score_t sc = (typename E::score_t)s;
+        score[grp] = sc;
+        if (sizeof(typename E::score_t) == 8) {
+            // Remember which key bits occur at all, so that radix passes over
+            // digits that are zero in every key can be skipped.
+            unsigned long long bits = (unsigned long long)sc;
+            unsigned long long seen = *reinterpret_cast<volatile unsigned long long *>(key_or);
+            if (bits & ~seen) atomicOr(key_or, bits);
+        }
+    }
+    // The first radix histogram is accumulated after this kernel; clear it here.
+    if (blockIdx.x == 0)
+        for (int i = threadIdx.x; i < hist0_len; i += kThreads) hist0[i] = 0;
+}
+
+// ---- a4 / a5: per-block perturbation over the lost set, optional restore ---
+
+template <typename T, int G, bool VEC, bool WRITE>
+__global__ void __launch_bounds__(kThreads)
+k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S,
+                 typename Elem<T>::score_t *__restrict__ part) {
+    using E = Elem<T>;
+    const int lane = threadIdx.x & (G - 1);
+    const uint64_t grp = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
+    const bool valid = grp < g.n_blocks && S.lost(g, (uint32_t)grp);
+    uint64_t beg = 0, len = 0;
+    if (valid) g.range((uint32_t)grp, beg, len);
+    typename E::wide_t s = block_distance<T, G, VEC, WRITE>(x, z, beg, len, lane);
+    if (valid && lane == 0) part[grp] = (typename E::score_t)s;
+}
+
+// ---- final reduction of the per-block partials in a fixed order -------------
+
+struct NormInfoDev {
+    double l2;
+    unsigned long long l1;
+    unsigned long long lost_blocks;
+    unsigned long long lost_elems;
+};
+
+constexpr int kReduceTile = 4096;  // blocks per CTA in the reduction
+
+template <typename W> __device__ __forceinline__ W cta_sum(W v, W *sh) {
+    v = group_sum<32, W>(v);
+    const int w = threadIdx.x >> 5;
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh[w] = v;
+    __syncthreads();
+    W t = 0;
+#pragma unroll
+    for (int i = 0; i < kThreads / 32; ++i) t += sh[i];
+    return t;
+}
+
+// Each CTA sums a fixed tile of per-block partials (fp64 for float data, exact
+// 64-bit for integer data) together with the lost block/element counts; the
+// CTA that finishes last adds the tile sums in tile order.  Which CTA is last
+// does not affect the order of any addition.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+k_reduce_partials(const typename Elem<T>::score_t *__restrict__ part, Geom g, LostSet S, double *tile_sum,
+                  unsigned long long *tile_l1, unsigned long long *tile_blocks, unsigned long long *tile_elems,
+                  unsigned *ticket, NormInfoDev *out) {
+    __shared__ double shd[kThreads / 32];
+    __shared__ unsigned long long shu[kThreads / 32];
+    __shared__ bool is_last;
+    const uint64_t base = (uint64_t)blockIdx.x * kReduceTile;
+    double fs = 0.0;
+    unsigned long long is = 0, nb = 0, ne = 0;
+    for (int j = 0; j < kReduceTile / kThreads; ++j) {
+        uint64_t b = base + threadIdx.x + (uint64_t)j * kThreads;
+        if (b < g.n_blocks && S.lost(g, (uint32_t)b)) {
+            uint64_t beg, len;
+            g.range((uint32_t)b, beg, len);
+            ++nb;
+            ne += len;
+            if (std::is_same<T, float>::value) fs += (double)part[b];
+            else is += (unsigned long long)part[b];
+        }
+    }
+    fs = cta_sum<double>(fs, shd);
+    is = cta_sum<unsigned long long>(is, shu);
+    nb = cta_sum<unsigned long long>(nb, shu);
+    ne = cta_sum<unsigned long long>(ne, shu);
+    if (threadIdx.x == 0) {
+        tile_sum[blockIdx.x] = fs;
+        tile_l1[blockIdx.x] = is;
+        tile_blocks[blockIdx.x] = nb;
+        tile_elems[blockIdx.x] = ne;
+        __threadfence();
+        is_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    fs = 0.0; is = 0; nb = 0; ne = 0;
+    for (unsigned t = threadIdx.x; t < gridDim.x; t += kThreads) {
+        fs += *reinterpret_cast<volatile double *>(tile_sum + t);
+        is += *reinterpret_cast<volatile unsigned long long *>(tile_l1 + t);
+        nb += *reinterpret_cast<volatile unsigned long long *>(tile_blocks + t);
+        ne += *reinterpret_cast<volatile unsigned long long *>(tile_elems + t);
+    }
+    fs = cta_sum<double>(fs, shd);
+    is = cta_sum<unsigned long long>(is, shu);
+    nb = cta_sum<unsigned long long>(nb, shu);
+    ne = cta_sum<unsigned long long>(ne, shu);
+    if (threadIdx.x == 0) {
+        out->l2 = sqrt(fs);
+        out->l1 = is;
+        out->lost_blocks = nb;
+        out->lost_elems = ne;
+        *ticket = 0;
+    }
+}
+
+// ---- plain copy (z := x at init, checkpoint reload) -------------------------
+
+__global__ void __launch_bounds__(kThreads)
+k_copy_elems(uint32_t *__restrict__ dst, const uint32_t *__restrict__ src, uint64_t n) {
+    const uint64_t nvec = n >> 2;
+    const uint64_t stride = (uint64_t)gridDim.x * kThreads;
+    uint4 *d4 = reinterpret_cast<uint4 *>(dst);
+    const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
+    for (uint64_t v = (uint64_t)blockIdx.x * kThreads + threadIdx.x; v < nvec; v += stride)
+        st_stream(d4 + v, ld_stream(s4 + v));
+    if (blockIdx.x == 0 && threadIdx.x < (n & 3)) dst[(nvec << 2) + threadIdx.x] = src[(nvec << 2) + threadIdx.x];
+}
+
+}  // namespace scar

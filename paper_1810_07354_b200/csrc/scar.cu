@@ -1,0 +1,648 @@
+// Host side of libscar: context, argument validation, launch sequencing and
+// the extern "C" entry points declared in include/scar.h.  Every step of the
+// checkpoint / recovery pass runs in the kernels of block_pass.cuh, select.cuh
+// and pack.cuh; there is no CPU path.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <type_traits>
+#include <vector>
+
+#include "scar.h"
+
+#include "block_pass.cuh"
+#include "pack.cuh"
+#include "select.cuh"
+
+using namespace scar;
+
+namespace {
+
+constexpr int kNumEvents = 6;
+
+}  // namespace
+
+struct scar_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    scar_dtype dt = SCAR_F32;
+    Geom g{};
+    int group_lanes = 32;
+
+    void *x = nullptr;  // caller-owned
+    void *z = nullptr;
+    void *payload = nullptr;
+    void *score = nullptr;  // float[B] or uint64[B]
+    void *part = nullptr;   // per-block perturbation partials, same type as score
+    uint32_t *sel = nullptr;
+    unsigned long long *poff = nullptr;
+    uint64_t *d_boff = nullptr;
+    uint8_t *d_shard_mask = nullptr;
+    SelState *st = nullptr;
+    TileArrays ta{};
+    unsigned n_sel_tiles = 0;
+    double *rt_sum = nullptr;
+    unsigned long long *rt_l1 = nullptr, *rt_blocks = nullptr, *rt_elems = nullptr;
+    unsigned n_red_tiles = 0;
+    SaveInfoDev *d_save = nullptr;
+    NormInfoDev *d_norm = nullptr;
+    SaveInfoDev *h_save = nullptr;  // pinned
+    NormInfoDev *h_norm = nullptr;  // pinned
+    bool have_save = false, have_norm = false;
+
+    std::vector<void *> owned;  // device allocations to free
+    uint64_t launches = 0;
+
+    bool profile = false;
+    cudaEvent_t ev[kNumEvents] = {};
+    int last_call = 0;  // 1 = save, 2 = recover / norm, 3 = scores only
+    bool ran_select = false, ran_pack = false;
+};
+
+namespace {
+
+#define CU_TRY(expr)                                  \
+    do {                                              \
+        cudaError_t e_ = (expr);                      \
+        if (e_ != cudaSuccess) return SCAR_ERR_CUDA;  \
+    } while (0)
+
+int check_device(const scar_ctx *c) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SCAR_ERR_CUDA;
+    return dev == c->device ? SCAR_OK : SCAR_ERR_STATE;
+}
+
+template <typename P> int dev_alloc(scar_ctx *c, P **p, size_t bytes) {
+    void *q = nullptr;
+    if (cudaMalloc(&q, bytes ? bytes : 16) != cudaSuccess) {
+        cudaGetLastError();
+        return SCAR_ERR_ALLOC;
+    }
+    c->owned.push_back(q);
+    *p = static_cast<P *>(q);
+    return SCAR_OK;
+}
+
+// Validates the caller's layout and fills the host-side fields of Geom
+// (boff is set later, once the offsets are on the device).
+int resolve_layout(const scar_layout *L, Geom &g) {
+    if (L->n_shards < 1) return SCAR_ERR_LAYOUT;
+    g = Geom{};
+    g.n_elems = L->n_elems;
+    g.n_shards = L->n_shards;
+    if (L->block_offsets) {
+        const uint64_t nb = L->n_blocks;
+        if (nb > 0xffffffffull - 1) return SCAR_ERR_LAYOUT;
+        const uint64_t *o = L->block_offsets;
+        if (o[0] != 0 || o[nb] != L->n_elems) return SCAR_ERR_LAYOUT;
+        bool vec = true;
+        for (uint64_t b = 0; b < nb; ++b) {
+            if (o[b + 1] < o[b]) return SCAR_ERR_LAYOUT;
+            if (o[b] & 3) vec = false;
+        }
+        if (o[nb] & 3) vec = false;
+        g.n_blocks = nb;
+        g.row_len = L->n_elems;
+        g.block_elems = 0;
+        g.blocks_per_row = 0;
+        g.vec_ok = vec;
+        return SCAR_OK;
+    }
+    if (L->n_elems == 0) {
+        g.n_blocks = 0;
+        g.row_len = 0;
+        g.block_elems = L->block_elems ? L->block_elems : 1;
+        g.blocks_per_row = 1;
+        g.vec_ok = 1;
+        return SCAR_OK;
+    }
+    if (L->block_elems == 0) return SCAR_ERR_LAYOUT;
+    const uint64_t row = L->row_elems ? L->row_elems : L->n_elems;
+    if (row > L->n_elems || L->n_elems % row != 0) return SCAR_ERR_LAYOUT;
+    const uint64_t per_row = (row + L->block_elems - 1) / L->block_elems;
+    const uint64_t rows = L->n_elems / row;
+    if (per_row > 0xfffffffeull || rows > 0xfffffffeull || per_row * rows > 0xfffffffeull) return SCAR_ERR_LAYOUT;
+    g.row_len = row;
+    g.block_elems = L->block_elems;
+    g.blocks_per_row = (uint32_t)per_row;
+    g.n_blocks = per_row * rows;
+    g.vec_ok = (row % 4 == 0) && (L->block_elems % 4 == 0);
+    return SCAR_OK;
+}
+
+// Lanes per block: about four 16-byte vectors (or four elements on the
+// element-wise path) per lane and stream, between 4 lanes and a full warp.
+int pick_group_lanes(const Geom &g) {
+    if (g.n_blocks == 0) return 32;
+    double units = (double)g.n_elems / (double)g.n_blocks;
+    if (g.vec_ok) units /= 4.0;
+    int G = 4;
+    while (G < 32 && G * 4 < units) G <<= 1;
+    return G;
+}
+
+template <typename F> void dispatch_group(int G, bool vec, F &&f) {
+    auto go = [&](auto gl) {
+        if (vec) f(gl, std::true_type{});
+        else f(gl, std::false_type{});
+    };
+    switch (G) {
+        case 4: go(std::integral_constant<int, 4>{}); break;
+        case 8: go(std::integral_constant<int, 8>{}); break;
+        case 16: go(std::integral_constant<int, 16>{}); break;
+        default: go(std::integral_constant<int, 32>{}); break;
+    }
+}
+
+unsigned grid_for_groups(uint64_t n_groups, int G) {
+    const uint64_t per_cta = kThreads / G;
+    return (unsigned)((n_groups + per_cta - 1) / per_cta);
+}
+
+void record(scar_ctx *c, int i) {
+    if (c->profile) cudaEventRecord(c->ev[i], c->stream);
+}
+
+// a1
+template <typename T> void launch_scores(scar_ctx *c) {
+    using S = typename Elem<T>::score_t;
+    if (c->g.n_blocks == 0) return;
+    dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
+        constexpr int G = decltype(gl)::value;
+        constexpr bool VEC = decltype(vec)::value;
+        k_block_scores<T, G, VEC><<<grid_for_groups(c->g.n_blocks, G), kThreads, 0, c->stream>>>(
+            static_cast<const T *>(c->x), static_cast<const T *>(c->z), c->g, static_cast<S *>(c->score),
+            &c->st->key_or, c->st->hist[0], kHistBins);
+    });
+    ++c->launches;
+}
+
+// a2
+template <typename K, typename S> void launch_select(scar_ctx *c, uint64_t k) {
+    using KT = KeyTraits<K>;
+    const unsigned nt = c->n_sel_tiles;
+    const S *score = static_cast<const S *>(c->score);
+    if (k > 0) {
+        for (int p = 0; p < KT::kPasses; ++p) {
+            k_radix_pass<K, S><<<nt, kThreads, 0, c->stream>>>(score, c->g.n_blocks, k, p, c->st);
+            ++c->launches;
+        }
+    }
+    k_select_count<K, S><<<nt, kThreads, 0, c->stream>>>(score, c->g, k, c->st, c->ta, c->d_save, c->poff);
+    ++c->launches;
+    if (k > 0) {
+        k_select_emit<K, S><<<nt, kThreads, 0, c->stream>>>(score, c->g, c->st, c->ta, c->sel, c->poff);
+        ++c->launches;
+    }
+}
+
+// a3
+void launch_pack(scar_ctx *c, uint64_t k) {
+    if (k == 0) return;
+    dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
+        constexpr int G = decltype(gl)::value;
+        constexpr bool VEC = decltype(vec)::value;
+        k_pack_update<G, VEC><<<grid_for_groups(k, G), kThreads, 0, c->stream>>>(
+            static_cast<const uint32_t *>(c->x), static_cast<uint32_t *>(c->z), static_cast<uint32_t *>(c->payload),
+            c->g, c->sel, c->poff, k);
+    });
+    ++c->launches;
+}
+
+// a4 / a5
+template <typename T> void launch_recover(scar_ctx *c, LostSet S, bool write) {
+    using Sc = typename Elem<T>::score_t;
+    dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
+        constexpr int G = decltype(gl)::value;
+        constexpr bool VEC = decltype(vec)::value;
+        const unsigned grid = grid_for_groups(c->g.n_blocks, G);
+        if (write)
+            k_recover_blocks<T, G, VEC, true><<<grid, kThreads, 0, c->stream>>>(
+                static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, static_cast<Sc *>(c->part));
+        else
+            k_recover_blocks<T, G, VEC, false><<<grid, kThreads, 0, c->stream>>>(
+                static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, static_cast<Sc *>(c->part));
+    });
+    ++c->launches;
+    record(c, 4);
+    k_reduce_partials<T><<<c->n_red_tiles, kThreads, 0, c->stream>>>(
+        static_cast<const Sc *>(c->part), c->g, S, c->rt_sum, c->rt_l1, c->rt_blocks, c->rt_elems,
+        &c->st->ticket_reduce, c->d_norm);
+    ++c->launches;
+    record(c, 5);
+}
+
+int copy_elems(scar_ctx *c, void *dst, const void *src, uint64_t n) {
+    if (n == 0) return SCAR_OK;
+    uint64_t want = ((n >> 2) + kThreads - 1) / kThreads;
+    unsigned grid = (unsigned)(want < 1 ? 1 : (want > 148u * 16u ? 148u * 16u : want));
+    k_copy_elems<<<grid, kThreads, 0, c->stream>>>(static_cast<uint32_t *>(dst), static_cast<const uint32_t *>(src), n);
+    ++c->launches;
+    CU_TRY(cudaGetLastError());
+    return SCAR_OK;
+}
+
+int fetch_save(scar_ctx *c, scar_save_info *out) {
+    CU_TRY(cudaMemcpyAsync(c->h_save, c->d_save, sizeof(SaveInfoDev), cudaMemcpyDeviceToHost, c->stream));
+    CU_TRY(cudaStreamSynchronize(c->stream));
+    out->k = c->h_save->k;
+    out->payload_elems = c->h_save->payload_elems;
+    out->nonfinite_blocks = c->h_save->nonfinite_blocks;
+    return SCAR_OK;
+}
+
+int fetch_norm(scar_ctx *c, scar_norm_info *out) {
+    CU_TRY(cudaMemcpyAsync(c->h_norm, c->d_norm, sizeof(NormInfoDev), cudaMemcpyDeviceToHost, c->stream));
+    CU_TRY(cudaStreamSynchronize(c->stream));
+    out->l2 = c->h_norm->l2;
+    out->l1 = c->h_norm->l1;
+    out->lost_blocks = c->h_norm->lost_blocks;
+    out->lost_elems = c->h_norm->lost_elems;
+    return SCAR_OK;
+}
+
+int k_from_r(double r, uint64_t n_blocks, uint64_t *k) {
+    if (!(r >= 0.0 && r <= 1.0)) return SCAR_ERR_INVALID_ARG;
+    long long v = llround(r * (double)n_blocks);
+    uint64_t kk = v < 0 ? 0 : (uint64_t)v;
+    if (kk > n_blocks) kk = n_blocks;
+    if (kk == 0 && r > 0.0 && n_blocks > 0) kk = 1;
+    *k = kk;
+    return SCAR_OK;
+}
+
+int enqueue_save(scar_ctx *c, uint64_t k) {
+    c->last_call = 1;
+    c->ran_select = c->ran_pack = false;
+    record(c, 0);
+    if (c->g.n_blocks == 0) {
+        CU_TRY(cudaMemsetAsync(c->d_save, 0, sizeof(SaveInfoDev), c->stream));
+        CU_TRY(cudaMemsetAsync(c->poff, 0, sizeof(unsigned long long), c->stream));
+        c->have_save = true;
+        return SCAR_OK;
+    }
+    if (c->dt == SCAR_F32) launch_scores<float>(c);
+    else launch_scores<int>(c);
+    record(c, 1);
+    if (c->dt == SCAR_F32) launch_select<unsigned, float>(c, k);
+    else launch_select<unsigned long long, unsigned long long>(c, k);
+    c->ran_select = true;
+    record(c, 2);
+    launch_pack(c, k);
+    c->ran_pack = k > 0;
+    record(c, 3);
+    CU_TRY(cudaGetLastError());
+    c->have_save = true;
+    return SCAR_OK;
+}
+
+int enqueue_recover(scar_ctx *c, LostSet S, bool write) {
+    c->last_call = 2;
+    record(c, 0);
+    if (c->g.n_blocks == 0) {
+        CU_TRY(cudaMemsetAsync(c->d_norm, 0, sizeof(NormInfoDev), c->stream));
+        c->have_norm = true;
+        return SCAR_OK;
+    }
+    if (c->dt == SCAR_F32) launch_recover<float>(c, S, write);
+    else launch_recover<int>(c, S, write);
+    CU_TRY(cudaGetLastError());
+    c->have_norm = true;
+    return SCAR_OK;
+}
+
+int shard_set(scar_ctx *c, const uint8_t *h_lost_shards, LostSet &S) {
+    CU_TRY(cudaMemcpyAsync(c->d_shard_mask, h_lost_shards, c->g.n_shards, cudaMemcpyHostToDevice, c->stream));
+    S.mask = c->d_shard_mask;
+    S.mode = 1;
+    return SCAR_OK;
+}
+
+void destroy_impl(scar_ctx *c) {
+    cudaStreamSynchronize(c->stream);
+    for (void *p : c->owned) cudaFree(p);
+    if (c->h_save) cudaFreeHost(c->h_save);
+    if (c->h_norm) cudaFreeHost(c->h_norm);
+    for (auto &e : c->ev)
+        if (e) cudaEventDestroy(e);
+    delete c;
+}
+
+}  // namespace
+
+extern "C" {
+
+int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *layout, void *cuda_stream) {
+    if (!out) return SCAR_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!layout || (dt != SCAR_F32 && dt != SCAR_I32)) return SCAR_ERR_INVALID_ARG;
+    if (layout->n_elems > 0 && !d_x) return SCAR_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_x) & 15) return SCAR_ERR_INVALID_ARG;
+    Geom g;
+    int rc = resolve_layout(layout, g);
+    if (rc != SCAR_OK) return rc;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return SCAR_ERR_CUDA;
+    }
+    scar_ctx *c = new (std::nothrow) scar_ctx;
+    if (!c) return SCAR_ERR_ALLOC;
+    c->device = dev;
+    c->stream = static_cast<cudaStream_t>(cuda_stream);
+    c->dt = dt;
+    c->g = g;
+    c->x = d_x;
+    c->group_lanes = pick_group_lanes(g);
+
+    const uint64_t N = g.n_elems, B = g.n_blocks;
+    const size_t score_bytes = (dt == SCAR_F32 ? 4 : 8) * B;
+    c->n_sel_tiles = (unsigned)((B + kSelTile - 1) / kSelTile);
+    if (c->n_sel_tiles == 0) c->n_sel_tiles = 1;
+    c->n_red_tiles = (unsigned)((B + kReduceTile - 1) / kReduceTile);
+    if (c->n_red_tiles == 0) c->n_red_tiles = 1;
+    const unsigned nt = c->n_sel_tiles, nr = c->n_red_tiles;
+
+    rc = SCAR_OK;
+    auto A = [&](auto **p, size_t bytes) {
+        if (rc == SCAR_OK) rc = dev_alloc(c, p, bytes);
+    };
+    A(&c->z, N * 4);
+    A(&c->payload, N * 4);
+    A(&c->score, score_bytes);
+    A(&c->part, score_bytes);
+    A(&c->sel, B * 4);
+    A(&c->poff, (B + 1) * 8);
+    A(&c->d_shard_mask, g.n_shards);
+    A(&c->st, sizeof(SelState));
+    A(&c->ta.gt, nt * 4);
+    A(&c->ta.eq, nt * 4);
+    A(&c->ta.nf, nt * 4);
+    A(&c->ta.len_gt, nt * 8);
+    A(&c->ta.len_eq, nt * 8);
+    A(&c->ta.eq_base, nt * 4);
+    A(&c->ta.sel_base, nt * 4);
+    A(&c->ta.len_base, nt * 8);
+    A(&c->rt_sum, nr * 8);
+    A(&c->rt_l1, nr * 8);
+    A(&c->rt_blocks, nr * 8);
+    A(&c->rt_elems, nr * 8);
+    A(&c->d_save, sizeof(SaveInfoDev));
+    A(&c->d_norm, sizeof(NormInfoDev));
+    if (rc == SCAR_OK && layout->block_offsets) A(&c->d_boff, (B + 1) * 8);
+    if (rc == SCAR_OK && (cudaMallocHost(&c->h_save, sizeof(SaveInfoDev)) != cudaSuccess ||
+                          cudaMallocHost(&c->h_norm, sizeof(NormInfoDev)) != cudaSuccess))
+        rc = SCAR_ERR_ALLOC;
+    if (rc == SCAR_OK) {
+        bool ok = cudaMemsetAsync(c->st, 0, sizeof(SelState), c->stream) == cudaSuccess &&
+                  cudaMemsetAsync(c->d_save, 0, sizeof(SaveInfoDev), c->stream) == cudaSuccess &&
+                  cudaMemsetAsync(c->d_norm, 0, sizeof(NormInfoDev), c->stream) == cudaSuccess &&
+                  cudaMemsetAsync(c->score, 0, score_bytes ? score_bytes : 16, c->stream) == cudaSuccess &&
+                  cudaMemsetAsync(c->poff, 0, 8, c->stream) == cudaSuccess;
+        if (ok && layout->block_offsets) {
+            ok = cudaMemcpyAsync(c->d_boff, layout->block_offsets, (B + 1) * 8, cudaMemcpyHostToDevice, c->stream) ==
+                 cudaSuccess;
+            c->g.boff = c->d_boff;
+        }
+        if (!ok) rc = SCAR_ERR_CUDA;
+    }
+    // Section 4.2: the running checkpoint starts as the initial parameter values.
+    if (rc == SCAR_OK) rc = copy_elems(c, c->z, c->x, N);
+    if (rc == SCAR_OK && cudaStreamSynchronize(c->stream) != cudaSuccess) rc = SCAR_ERR_CUDA;
+    if (rc != SCAR_OK) {
+        cudaGetLastError();
+        destroy_impl(c);
+        return rc;
+    }
+    *out = c;
+    return SCAR_OK;
+}
+
+int scar_ckpt_block_scores(scar_ctx *c) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    c->last_call = 3;
+    record(c, 0);
+    if (c->dt == SCAR_F32) launch_scores<float>(c);
+    else launch_scores<int>(c);
+    record(c, 1);
+    CU_TRY(cudaGetLastError());
+    return SCAR_OK;
+}
+
+int scar_ckpt_priority_save_k(scar_ctx *c, uint64_t k, scar_save_info *out) {
+    if (!c || k > c->g.n_blocks) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    rc = enqueue_save(c, k);
+    if (rc != SCAR_OK) return rc;
+    return out ? fetch_save(c, out) : SCAR_OK;
+}
+
+int scar_ckpt_priority_save(scar_ctx *c, double r, scar_save_info *out) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    uint64_t k = 0;
+    int rc = k_from_r(r, c->g.n_blocks, &k);
+    if (rc != SCAR_OK) return rc;
+    return scar_ckpt_priority_save_k(c, k, out);
+}
+
+int scar_recover_partial(scar_ctx *c, const uint8_t *h_lost_shards, scar_norm_info *out) {
+    if (!c || !h_lost_shards) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    LostSet S{};
+    rc = shard_set(c, h_lost_shards, S);
+    if (rc == SCAR_OK) rc = enqueue_recover(c, S, true);
+    if (rc != SCAR_OK) return rc;
+    return out ? fetch_norm(c, out) : SCAR_OK;
+}
+
+int scar_recover_partial_blocks(scar_ctx *c, const uint8_t *d_lost_blocks, scar_norm_info *out) {
+    if (!c || (!d_lost_blocks && c->g.n_blocks)) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    LostSet S{d_lost_blocks, 2};
+    rc = enqueue_recover(c, S, true);
+    if (rc != SCAR_OK) return rc;
+    return out ? fetch_norm(c, out) : SCAR_OK;
+}
+
+int scar_perturbation_norm(scar_ctx *c, const uint8_t *h_lost_shards, scar_norm_info *out) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    LostSet S{nullptr, 0};
+    if (h_lost_shards) rc = shard_set(c, h_lost_shards, S);
+    if (rc == SCAR_OK) rc = enqueue_recover(c, S, false);
+    if (rc != SCAR_OK) return rc;
+    return out ? fetch_norm(c, out) : SCAR_OK;
+}
+
+int scar_perturbation_norm_blocks(scar_ctx *c, const uint8_t *d_lost_blocks, scar_norm_info *out) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    LostSet S{d_lost_blocks, d_lost_blocks ? 2 : 0};
+    rc = enqueue_recover(c, S, false);
+    if (rc != SCAR_OK) return rc;
+    return out ? fetch_norm(c, out) : SCAR_OK;
+}
+
+int scar_ckpt_priority_save_host(scar_ctx *c, const void *h_x, double r, void *h_payload, uint32_t *h_sel,
+                                 uint64_t *h_poff, scar_save_info *out) {
+    if (!c || !out || !h_poff) return SCAR_ERR_INVALID_ARG;
+    const uint64_t N = c->g.n_elems;
+    uint64_t k = 0;
+    int rc = k_from_r(r, c->g.n_blocks, &k);
+    if (rc != SCAR_OK) return rc;
+    if (N && (!h_x || !h_payload)) return SCAR_ERR_INVALID_ARG;
+    if (k && !h_sel) return SCAR_ERR_INVALID_ARG;
+    rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    if (N) CU_TRY(cudaMemcpyAsync(c->x, h_x, N * 4, cudaMemcpyHostToDevice, c->stream));
+    rc = enqueue_save(c, k);
+    if (rc != SCAR_OK) return rc;
+    // The id and offset lists have a size known up front; the payload length is data dependent.
+    if (k) CU_TRY(cudaMemcpyAsync(h_sel, c->sel, k * 4, cudaMemcpyDeviceToHost, c->stream));
+    CU_TRY(cudaMemcpyAsync(h_poff, c->poff, (k + 1) * 8, cudaMemcpyDeviceToHost, c->stream));
+    rc = fetch_save(c, out);
+    if (rc != SCAR_OK) return rc;
+    if (out->payload_elems) {
+        CU_TRY(cudaMemcpyAsync(h_payload, c->payload, out->payload_elems * 4, cudaMemcpyDeviceToHost, c->stream));
+        CU_TRY(cudaStreamSynchronize(c->stream));
+    }
+    return SCAR_OK;
+}
+
+int scar_recover_partial_host(scar_ctx *c, void *h_x, const uint8_t *h_lost_shards, scar_norm_info *out) {
+    if (!c || !h_lost_shards || !out) return SCAR_ERR_INVALID_ARG;
+    if (c->g.n_elems && !h_x) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    // Element range of every lost shard, from the block offsets the library resolved.
+    const uint64_t B = c->g.n_blocks, S = c->g.n_shards;
+    std::vector<uint64_t> lo, hi;
+    auto elem_of = [&](uint64_t b, uint64_t &e) -> int {
+        if (b >= B) { e = c->g.n_elems; return SCAR_OK; }
+        if (c->g.boff) {
+            CU_TRY(cudaMemcpyAsync(&e, c->g.boff + b, 8, cudaMemcpyDeviceToHost, c->stream));
+            CU_TRY(cudaStreamSynchronize(c->stream));
+            return SCAR_OK;
+        }
+        uint64_t row = b / c->g.blocks_per_row, j = b % c->g.blocks_per_row;
+        e = row * c->g.row_len + j * c->g.block_elems;
+        return SCAR_OK;
+    };
+    for (uint64_t s = 0; s < S && B; ++s) {
+        if (!h_lost_shards[s]) continue;
+        uint64_t b0 = (uint64_t)(((unsigned __int128)s * B) / S), b1 = (uint64_t)(((unsigned __int128)(s + 1) * B) / S);
+        if (b0 == b1) continue;
+        uint64_t e0, e1;
+        if ((rc = elem_of(b0, e0)) != SCAR_OK || (rc = elem_of(b1, e1)) != SCAR_OK) return rc;
+        if (!lo.empty() && hi.back() == e0) hi.back() = e1;
+        else { lo.push_back(e0); hi.push_back(e1); }
+    }
+    char *hx = static_cast<char *>(h_x), *dx = static_cast<char *>(c->x);
+    for (size_t i = 0; i < lo.size(); ++i)
+        CU_TRY(cudaMemcpyAsync(dx + lo[i] * 4, hx + lo[i] * 4, (hi[i] - lo[i]) * 4, cudaMemcpyHostToDevice, c->stream));
+    LostSet Ls{};
+    rc = shard_set(c, h_lost_shards, Ls);
+    if (rc == SCAR_OK) rc = enqueue_recover(c, Ls, true);
+    if (rc != SCAR_OK) return rc;
+    for (size_t i = 0; i < lo.size(); ++i)
+        CU_TRY(cudaMemcpyAsync(hx + lo[i] * 4, dx + lo[i] * 4, (hi[i] - lo[i]) * 4, cudaMemcpyDeviceToHost, c->stream));
+    return fetch_norm(c, out);
+}
+
+int scar_ckpt_load(scar_ctx *c, const void *d_z_src) {
+    if (!c || (!d_z_src && c->g.n_elems)) return SCAR_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_z_src) & 15) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    return copy_elems(c, c->z, d_z_src, c->g.n_elems);
+}
+
+int scar_ckpt_last_info(scar_ctx *c, scar_save_info *save, scar_norm_info *norm) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    if ((save && !c->have_save) || (norm && !c->have_norm)) return SCAR_ERR_STATE;
+    if (save && (rc = fetch_save(c, save)) != SCAR_OK) return rc;
+    if (norm && (rc = fetch_norm(c, norm)) != SCAR_OK) return rc;
+    if (!save && !norm) CU_TRY(cudaStreamSynchronize(c->stream));
+    return SCAR_OK;
+}
+
+int scar_ckpt_view(scar_ctx *c, const void **d_z, const void **d_scores, const uint32_t **d_sel,
+                   const uint64_t **d_poff, const void **d_payload) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    if (d_z) *d_z = c->z;
+    if (d_scores) *d_scores = c->score;
+    if (d_sel) *d_sel = c->sel;
+    if (d_poff) *d_poff = reinterpret_cast<const uint64_t *>(c->poff);
+    if (d_payload) *d_payload = c->payload;
+    return SCAR_OK;
+}
+
+uint64_t scar_ckpt_n_blocks(const scar_ctx *c) { return c ? c->g.n_blocks : 0; }
+
+uint64_t scar_ckpt_launch_count(const scar_ctx *c) { return c ? c->launches : 0; }
+
+int scar_ckpt_profile(scar_ctx *c, int enable) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    if (enable && !c->ev[0])
+        for (auto &e : c->ev) CU_TRY(cudaEventCreate(&e));
+    c->profile = enable != 0;
+    c->last_call = 0;
+    return SCAR_OK;
+}
+
+int scar_ckpt_profile_read(scar_ctx *c, float ms[5]) {
+    if (!c || !ms) return SCAR_ERR_INVALID_ARG;
+    if (!c->profile) return SCAR_ERR_STATE;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    for (int i = 0; i < 5; ++i) ms[i] = 0.f;
+    CU_TRY(cudaStreamSynchronize(c->stream));
+    if (c->g.n_blocks == 0) return SCAR_OK;
+    if (c->last_call == 1 || c->last_call == 3) {
+        CU_TRY(cudaEventElapsedTime(&ms[0], c->ev[0], c->ev[1]));
+        if (c->last_call == 1) {
+            CU_TRY(cudaEventElapsedTime(&ms[1], c->ev[1], c->ev[2]));
+            CU_TRY(cudaEventElapsedTime(&ms[2], c->ev[2], c->ev[3]));
+        }
+    } else if (c->last_call == 2) {
+        CU_TRY(cudaEventElapsedTime(&ms[3], c->ev[0], c->ev[4]));
+        CU_TRY(cudaEventElapsedTime(&ms[4], c->ev[4], c->ev[5]));
+    }
+    return SCAR_OK;
+}
+
+int scar_ckpt_destroy(scar_ctx *c) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    destroy_impl(c);
+    return SCAR_OK;
+}
+
+const char *scar_strerror(int code) {
+    switch (code) {
+        case SCAR_OK: return "ok";
+        case SCAR_ERR_INVALID_ARG: return "invalid argument";
+        case SCAR_ERR_LAYOUT: return "inconsistent block layout";
+        case SCAR_ERR_ALLOC: return "allocation failed";
+        case SCAR_ERR_CUDA: return "CUDA runtime error";
+        case SCAR_ERR_STATE: return "call not valid in this state";
+        case SCAR_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"
