@@ -196,7 +196,7 @@ def cpu_baseline(x_dev, z_dev, lost_shards):
     """Times the oracle on a prefix of the device-resident workload (copied to the host)."""
     import oracle
 
-    n = 1 << 27
+    n = min(x_dev.numel(), 1 << 30)
     nb = n // BLOCK
     x = x_dev[:n].cpu().numpy()
     z = z_dev[:n].cpu().numpy()
@@ -204,7 +204,7 @@ def cpu_baseline(x_dev, z_dev, lost_shards):
     lost = oracle.expand_shards(nb, lost_shards)
     t_save, _ = oracle_step(x, z, boff, lost, {})
     return {"value": len(R_SWEEP) * 2 * n * ELEM / t_save / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"one step on the first {n} of {N_ELEMS} elements ({nb} blocks) of the same buffers, "
+            "sample": f"one step on {n} of {N_ELEMS} elements ({nb} blocks) of the same buffers, "
                       f"single thread, {t_save:.1f} s in saves"}
 
 

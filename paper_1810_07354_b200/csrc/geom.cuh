@@ -42,14 +42,32 @@ struct Geom {
     }
 };
 
-// How a kernel decides whether block b belongs to the lost set S.
+// The lost set S of a recovery (Section 4.1), as a list of work items that the
+// recovery kernels map to blocks.
+//   mode 0: every block is lost; work item w is block w.
+//   mode 1: runs of consecutive lost blocks (lost shards, adjacent ones merged);
+//           only lost blocks are work items, so no CTA is launched for the rest.
+//   mode 2: per-block mask in device memory; work item w is block w, skipped
+//           when mask[w] == 0.
+constexpr int kMaxRuns = 32;
 struct LostSet {
-    const uint8_t *mask;  // per shard (mode 1) or per block (mode 2); unused in mode 0
-    int mode;             // 0: every block lost, 1: shard mask, 2: block mask
-    __device__ __forceinline__ bool lost(const Geom &g, uint32_t b) const {
-        if (mode == 0) return true;
-        if (mode == 1) return mask[g.shard_of(b)] != 0;
-        return mask[b] != 0;
+    const uint8_t *mask;
+    uint64_t n_work;
+    int mode;
+    int n_runs;
+    uint32_t run_first[kMaxRuns];      // first block of run r
+    uint32_t run_start[kMaxRuns + 1];  // work items before run r
+
+    __device__ __forceinline__ bool block_of(uint64_t w, uint32_t &b) const {
+        if (w >= n_work) return false;
+        if (mode == 1) {
+            int r = 0;
+            while (r + 1 < n_runs && w >= run_start[r + 1]) ++r;
+            b = run_first[r] + (uint32_t)(w - run_start[r]);
+            return true;
+        }
+        b = (uint32_t)w;
+        return mode == 0 || mask[b] != 0;
     }
 };
 

@@ -7,6 +7,44 @@
 
 namespace scar {
 
+// A group of G lanes copies one selected block, four units per lane and batch,
+// with the loads of the next batch issued before the stores of the current one
+// (see block_distance for why).
+template <typename U, int G>
+__device__ __forceinline__ void copy_block_2dst(const U *__restrict__ src, U *__restrict__ d0, U *__restrict__ d1,
+                                                uint64_t n, int lane) {
+    constexpr uint64_t step = 4 * (uint64_t)G;
+    U c[4], nx[4];
+    uint64_t u = lane;
+    bool have = u < n;
+    if (have) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (u + (uint64_t)j * G < n) c[j] = ld_stream(src + u + (uint64_t)j * G);
+    }
+    while (have) {
+        const uint64_t un = u + step;
+        const bool more = un < n;
+        if (more) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (un + (uint64_t)j * G < n) nx[j] = ld_stream(src + un + (uint64_t)j * G);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint64_t i = u + (uint64_t)j * G;
+            if (i < n) {
+                st_stream(d0 + i, c[j]);
+                st_stream(d1 + i, c[j]);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) c[j] = nx[j];
+        u = un;
+        have = more;
+    }
+}
+
 template <int G, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 k_pack_update(const uint32_t *__restrict__ x, uint32_t *__restrict__ z, uint32_t *__restrict__ payload, Geom g,
@@ -17,39 +55,11 @@ k_pack_update(const uint32_t *__restrict__ x, uint32_t *__restrict__ z, uint32_t
     uint64_t beg, len;
     g.range(sel[j], beg, len);
     const uint64_t dst = poff[j];
-    if (VEC) {
-        const uint4 *xv = reinterpret_cast<const uint4 *>(x + beg);
-        uint4 *zv = reinterpret_cast<uint4 *>(z + beg);
-        uint4 *pv = reinterpret_cast<uint4 *>(payload + dst);
-        const uint64_t nvec = len >> 2;
-        uint64_t v = lane;
-        for (; v + 3 * G < nvec; v += 4 * G) {
-            uint4 a = ld_stream(xv + v), b = ld_stream(xv + v + G), c = ld_stream(xv + v + 2 * G),
-                  d = ld_stream(xv + v + 3 * G);
-            st_stream(pv + v, a); st_stream(pv + v + G, b); st_stream(pv + v + 2 * G, c); st_stream(pv + v + 3 * G, d);
-            st_stream(zv + v, a); st_stream(zv + v + G, b); st_stream(zv + v + 2 * G, c); st_stream(zv + v + 3 * G, d);
-        }
-        for (; v < nvec; v += G) {
-            uint4 a = ld_stream(xv + v);
-            st_stream(pv + v, a);
-            st_stream(zv + v, a);
-        }
-    } else {
-        const uint32_t *xs = x + beg;
-        uint32_t *zs = z + beg, *ps = payload + dst;
-        uint64_t i = lane;
-        for (; i + 3 * G < len; i += 4 * G) {
-            uint32_t a = ld_stream(xs + i), b = ld_stream(xs + i + G), c = ld_stream(xs + i + 2 * G),
-                     d = ld_stream(xs + i + 3 * G);
-            ps[i] = a; ps[i + G] = b; ps[i + 2 * G] = c; ps[i + 3 * G] = d;
-            zs[i] = a; zs[i + G] = b; zs[i + 2 * G] = c; zs[i + 3 * G] = d;
-        }
-        for (; i < len; i += G) {
-            uint32_t a = ld_stream(xs + i);
-            ps[i] = a;
-            zs[i] = a;
-        }
-    }
+    if (VEC)
+        copy_block_2dst<uint4, G>(reinterpret_cast<const uint4 *>(x + beg), reinterpret_cast<uint4 *>(payload + dst),
+                                  reinterpret_cast<uint4 *>(z + beg), len >> 2, lane);
+    else
+        copy_block_2dst<uint32_t, G>(x + beg, payload + dst, z + beg, len, lane);
 }
 
 }  // namespace scar

@@ -40,6 +40,7 @@ struct scar_ctx {
     unsigned long long *poff = nullptr;
     uint64_t *d_boff = nullptr;
     uint8_t *d_shard_mask = nullptr;
+    uint8_t *d_block_mask = nullptr;  // only used when a shard mask has too many runs
     SelState *st = nullptr;
     TileArrays ta{};
     unsigned n_sel_tiles = 0;
@@ -213,22 +214,26 @@ void launch_pack(scar_ctx *c, uint64_t k) {
 }
 
 // a4 / a5
-template <typename T> void launch_recover(scar_ctx *c, LostSet S, bool write) {
+template <typename T> void launch_recover(scar_ctx *c, const LostSet &S, bool write) {
     using Sc = typename Elem<T>::score_t;
-    dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
-        constexpr int G = decltype(gl)::value;
-        constexpr bool VEC = decltype(vec)::value;
-        const unsigned grid = grid_for_groups(c->g.n_blocks, G);
-        if (write)
-            k_recover_blocks<T, G, VEC, true><<<grid, kThreads, 0, c->stream>>>(
-                static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, static_cast<Sc *>(c->part));
-        else
-            k_recover_blocks<T, G, VEC, false><<<grid, kThreads, 0, c->stream>>>(
-                static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, static_cast<Sc *>(c->part));
-    });
-    ++c->launches;
+    if (S.n_work > 0) {
+        dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
+            constexpr int G = decltype(gl)::value;
+            constexpr bool VEC = decltype(vec)::value;
+            const unsigned grid = grid_for_groups(S.n_work, G);
+            if (write)
+                k_recover_blocks<T, G, VEC, true><<<grid, kThreads, 0, c->stream>>>(
+                    static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, static_cast<Sc *>(c->part));
+            else
+                k_recover_blocks<T, G, VEC, false><<<grid, kThreads, 0, c->stream>>>(
+                    static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, static_cast<Sc *>(c->part));
+        });
+        ++c->launches;
+    }
     record(c, 4);
-    k_reduce_partials<T><<<c->n_red_tiles, kThreads, 0, c->stream>>>(
+    uint64_t tiles = (S.n_work + kReduceTile - 1) / kReduceTile;
+    if (tiles == 0) tiles = 1;
+    k_reduce_partials<T><<<(unsigned)tiles, kThreads, 0, c->stream>>>(
         static_cast<const Sc *>(c->part), c->g, S, c->rt_sum, c->rt_l1, c->rt_blocks, c->rt_elems,
         &c->st->ticket_reduce, c->d_norm);
     ++c->launches;
@@ -299,7 +304,7 @@ int enqueue_save(scar_ctx *c, uint64_t k) {
     return SCAR_OK;
 }
 
-int enqueue_recover(scar_ctx *c, LostSet S, bool write) {
+int enqueue_recover(scar_ctx *c, const LostSet &S, bool write) {
     c->last_call = 2;
     record(c, 0);
     if (c->g.n_blocks == 0) {
@@ -314,10 +319,57 @@ int enqueue_recover(scar_ctx *c, LostSet S, bool write) {
     return SCAR_OK;
 }
 
+LostSet all_lost(const scar_ctx *c) {
+    LostSet S{};
+    S.mode = 0;
+    S.n_work = c->g.n_blocks;
+    return S;
+}
+
+LostSet block_mask_set(const scar_ctx *c, const uint8_t *d_lost_blocks) {
+    LostSet S{};
+    S.mode = 2;
+    S.mask = d_lost_blocks;
+    S.n_work = c->g.n_blocks;
+    return S;
+}
+
+// Lost shards -> runs of consecutive lost blocks (adjacent lost shards merge,
+// shards that own no block vanish).  With more runs than LostSet can carry,
+// the shard mask is expanded into a per-block mask on the device instead.
 int shard_set(scar_ctx *c, const uint8_t *h_lost_shards, LostSet &S) {
-    CU_TRY(cudaMemcpyAsync(c->d_shard_mask, h_lost_shards, c->g.n_shards, cudaMemcpyHostToDevice, c->stream));
-    S.mask = c->d_shard_mask;
+    const uint64_t B = c->g.n_blocks, n_sh = c->g.n_shards;
+    S = LostSet{};
     S.mode = 1;
+    bool overflow = false;
+    uint64_t work = 0;
+    for (uint64_t s = 0; s < n_sh && B; ++s) {
+        if (!h_lost_shards[s]) continue;
+        const uint64_t lo = (uint64_t)(((unsigned __int128)s * B) / n_sh);
+        const uint64_t hi = (uint64_t)(((unsigned __int128)(s + 1) * B) / n_sh);
+        if (lo == hi) continue;
+        if (S.n_runs > 0 && (uint64_t)S.run_first[S.n_runs - 1] + (work - S.run_start[S.n_runs - 1]) == lo) {
+            work += hi - lo;  // extends the previous run
+        } else {
+            if (S.n_runs == kMaxRuns) {
+                overflow = true;
+                break;
+            }
+            S.run_first[S.n_runs] = (uint32_t)lo;
+            S.run_start[S.n_runs] = (uint32_t)work;
+            ++S.n_runs;
+            work += hi - lo;
+        }
+        S.run_start[S.n_runs] = (uint32_t)work;
+    }
+    S.n_work = work;
+    if (!overflow) return SCAR_OK;
+    CU_TRY(cudaMemcpyAsync(c->d_shard_mask, h_lost_shards, n_sh, cudaMemcpyHostToDevice, c->stream));
+    k_expand_shards<<<(unsigned)((B + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(c->g, c->d_shard_mask,
+                                                                                          c->d_block_mask);
+    ++c->launches;
+    CU_TRY(cudaGetLastError());
+    S = block_mask_set(c, c->d_block_mask);
     return SCAR_OK;
 }
 
@@ -378,6 +430,7 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     A(&c->sel, B * 4);
     A(&c->poff, (B + 1) * 8);
     A(&c->d_shard_mask, g.n_shards);
+    A(&c->d_block_mask, B);
     A(&c->st, sizeof(SelState));
     A(&c->ta.gt, nt * 4);
     A(&c->ta.eq, nt * 4);
@@ -467,7 +520,7 @@ int scar_recover_partial_blocks(scar_ctx *c, const uint8_t *d_lost_blocks, scar_
     if (!c || (!d_lost_blocks && c->g.n_blocks)) return SCAR_ERR_INVALID_ARG;
     int rc = check_device(c);
     if (rc != SCAR_OK) return rc;
-    LostSet S{d_lost_blocks, 2};
+    LostSet S = block_mask_set(c, d_lost_blocks);
     rc = enqueue_recover(c, S, true);
     if (rc != SCAR_OK) return rc;
     return out ? fetch_norm(c, out) : SCAR_OK;
@@ -477,7 +530,7 @@ int scar_perturbation_norm(scar_ctx *c, const uint8_t *h_lost_shards, scar_norm_
     if (!c) return SCAR_ERR_INVALID_ARG;
     int rc = check_device(c);
     if (rc != SCAR_OK) return rc;
-    LostSet S{nullptr, 0};
+    LostSet S = all_lost(c);
     if (h_lost_shards) rc = shard_set(c, h_lost_shards, S);
     if (rc == SCAR_OK) rc = enqueue_recover(c, S, false);
     if (rc != SCAR_OK) return rc;
@@ -488,7 +541,7 @@ int scar_perturbation_norm_blocks(scar_ctx *c, const uint8_t *d_lost_blocks, sca
     if (!c) return SCAR_ERR_INVALID_ARG;
     int rc = check_device(c);
     if (rc != SCAR_OK) return rc;
-    LostSet S{d_lost_blocks, d_lost_blocks ? 2 : 0};
+    LostSet S = d_lost_blocks ? block_mask_set(c, d_lost_blocks) : all_lost(c);
     rc = enqueue_recover(c, S, false);
     if (rc != SCAR_OK) return rc;
     return out ? fetch_norm(c, out) : SCAR_OK;

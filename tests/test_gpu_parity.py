@@ -275,6 +275,30 @@ def test_masks_empty_full_and_more_shards_than_blocks():
     ck.close()
 
 
+@pytest.mark.parametrize("n_shards,pattern", [(100, "alternate"), (64, "pairs"), (33, "alternate"), (7, "ends")])
+def test_many_lost_shard_runs(n_shards, pattern):
+    # few runs travel inside the launch parameters, many fall back to a device-side block mask
+    w = make_workload("tiny", n_elems=1 << 18, block_elems=64)  # 4096 blocks
+    boff = block_offsets(w.geom)
+    m = np.zeros(n_shards, dtype=np.uint8)
+    if pattern == "alternate":
+        m[::2] = 1
+    elif pattern == "pairs":
+        m[0::4] = 1
+        m[1::4] = 1
+    else:
+        m[0] = m[-1] = 1
+    xd = parity.to_dev(w.x)
+    ck = api.ScarCheckpoint(xd, n_shards=n_shards, block_elems=64)
+    ck.load(parity.to_dev(w.z))
+    lb = oracle.expand_shards(w.n_blocks, m)
+    ora_n, x_after = oracle.recover_partial(w.x, w.z, boff, lb)
+    parity.check_norm(ck.perturbation_norm(m), ora_n, True)
+    parity.check_norm(ck.recover_partial(m), ora_n, True)
+    assert xd.cpu().numpy().tobytes() == x_after.tobytes()
+    ck.close()
+
+
 def test_recovery_does_not_write_outside_x():
     w = make_workload("mf", l_rows=4000, r_rows=150)
     n = w.x.size
