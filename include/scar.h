@@ -50,7 +50,8 @@ enum {
     SCAR_ERR_ALLOC = -3,       /* device or host allocation failed */
     SCAR_ERR_CUDA = -4,        /* a CUDA runtime call or kernel launch failed */
     SCAR_ERR_STATE = -5,       /* call not valid in the context's current state */
-    SCAR_ERR_TIMEOUT = -6      /* reserved: a bounded device-side wait gave up */
+    SCAR_ERR_TIMEOUT = -6,     /* reserved: a bounded device-side wait gave up */
+    SCAR_ERR_CAPACITY = -7     /* problem larger than a fixed-size internal buffer */
 };
 
 /* Block geometry of the flat buffer of n_elems elements.
@@ -127,6 +128,36 @@ int scar_recover_partial_blocks(scar_ctx *ctx, const uint8_t *d_lost_blocks, sca
  * perturbation is x^(T) - x^(C) (Example 2.3). */
 int scar_perturbation_norm(scar_ctx *ctx, const uint8_t *h_lost_shards, scar_norm_info *out);
 int scar_perturbation_norm_blocks(scar_ctx *ctx, const uint8_t *d_lost_blocks, scar_norm_info *out);
+
+/* Perturbation norm without any allocation.  (The paper has no counterpart: it
+ * is the same quantity as scar_perturbation_norm_blocks, offered for callers
+ * that cannot allocate.)
+ *
+ * Some callers cannot create a context, because scar_ckpt_init calls cudaMalloc:
+ * a failure handler running while memory is exhausted, a latency-critical loop
+ * that cannot take the device-wide synchronisation an allocation implies, or a
+ * plug-in whose host forbids it to grow its memory.  This call needs no
+ * context and calls no cudaMalloc / cudaFree or other allocating routine.  Its
+ * per-block partial sums live in a fixed array of about 8 MiB inside the
+ * library's device image (every GPU that loads the library holds it until the
+ * process exits), which caps the problem at SCAR_STATIC_MAX_BLOCKS blocks;
+ * larger layouts return SCAR_ERR_CAPACITY and nothing is enqueued.
+ *
+ *   d_x, d_z       DEVICE buffers of layout->n_elems elements of type dt, both
+ *                  16-byte aligned, read only; z is the checkpoint to compare with
+ *   layout         implicit form only (block_offsets must be NULL); n_shards ignored
+ *   d_lost_blocks  DEVICE array of B bytes, 0 alive / non-zero lost; NULL = all lost
+ *   d_out          DEVICE scar_norm_info written by the enqueued work (caller-owned)
+ *   cuda_stream    cudaStream_t to enqueue on; the call does not wait
+ *
+ * The first call on each device looks up the array's device address (once, with
+ * that device current); make that first call before any stream capture.  All
+ * calls on a device share the one array: calls whose GPU work overlaps (different
+ * streams, or different threads) race and give wrong results; calls ordered on
+ * one stream are fine.  Results are bit-identical to scar_perturbation_norm_blocks. */
+#define SCAR_STATIC_MAX_BLOCKS (1ull << 20)
+int scar_perturbation_norm_static(const void *d_x, const void *d_z, scar_dtype dt, const scar_layout *layout,
+                                  const uint8_t *d_lost_blocks, scar_norm_info *d_out, void *cuda_stream);
 
 /* Host-buffer forms for callers whose parameters live in host memory.
  * save_host: copies n_elems elements from h_x into the context's x, runs the

@@ -27,14 +27,15 @@ def is_stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile ``csrc/scar.cu`` into ``libscar.so`` next to this file if it is missing or out of date."""
+    """Compile ``csrc/*.cu`` into ``libscar.so`` next to this file if it is missing or out of date."""
     if not force and not is_stale():
         return LIB
     nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
     if not os.path.exists(nvcc):
         raise RuntimeError("nvcc not found: libscar.so cannot be built")
     tmp = f"{LIB}.{os.getpid()}.tmp"
-    cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-o", tmp, os.path.join(CSRC, "scar.cu")]
+    units = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cu"))
+    cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-o", tmp, *units]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     subprocess.check_call(cmd)

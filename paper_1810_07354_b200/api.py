@@ -64,6 +64,7 @@ _SIGS = {
     "scar_recover_partial_blocks": (_int, [_vp, _vp, C.POINTER(scar_norm_info)]),
     "scar_perturbation_norm": (_int, [_vp, _vp, C.POINTER(scar_norm_info)]),
     "scar_perturbation_norm_blocks": (_int, [_vp, _vp, C.POINTER(scar_norm_info)]),
+    "scar_perturbation_norm_static": (_int, [_vp, _vp, _int, C.POINTER(scar_layout), _vp, _vp, _vp]),
     "scar_ckpt_priority_save_host": (_int, [_vp, _vp, _dbl, _vp, _vp, _vp, C.POINTER(scar_save_info)]),
     "scar_recover_partial_host": (_int, [_vp, _vp, _vp, C.POINTER(scar_norm_info)]),
     "scar_ckpt_load": (_int, [_vp, _vp]),
@@ -180,6 +181,15 @@ def scar_perturbation_norm(ctx: int, h_lost_shards: Optional[np.ndarray] = None,
 
 def scar_perturbation_norm_blocks(ctx: int, d_lost_blocks=None, sync: bool = True):
     return _norm_call("scar_perturbation_norm_blocks", ctx, d_lost_blocks, sync)
+
+
+def scar_perturbation_norm_static(d_x, d_z, dtype: int, layout: scar_layout, d_lost_blocks, d_out,
+                                  cuda_stream: int = 0) -> None:
+    """Allocation-free perturbation norm: enqueues on ``cuda_stream`` and writes a ``scar_norm_info`` to the
+    caller's device buffer ``d_out`` (32 bytes).  See ``include/scar.h`` for who needs it and its limits."""
+    _check(load_library().scar_perturbation_norm_static(_addr(d_x), _addr(d_z), dtype, C.byref(layout),
+                                                        _addr(d_lost_blocks), _addr(d_out), cuda_stream or None),
+           "scar_perturbation_norm_static")
 
 
 def scar_ckpt_priority_save_host(ctx: int, h_x, r: float, h_payload, h_sel, h_poff) -> scar_save_info:

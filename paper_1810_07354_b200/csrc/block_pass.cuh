@@ -213,7 +213,7 @@ k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S,
 }
 
 // Lost shards as a per-block mask, for lost sets with more runs than LostSet holds.
-__global__ void __launch_bounds__(kThreads)
+static __global__ void __launch_bounds__(kThreads)
 k_expand_shards(Geom g, const uint8_t *__restrict__ shard_mask, uint8_t *__restrict__ block_mask) {
     const uint64_t b = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
     if (b < g.n_blocks) block_mask[b] = shard_mask[g.shard_of((uint32_t)b)] != 0;
@@ -312,7 +312,7 @@ k_reduce_partials(const typename Elem<T>::score_t *__restrict__ part, Geom g, Lo
 
 // ---- plain copy (z := x at init, checkpoint reload) -------------------------
 
-__global__ void __launch_bounds__(kThreads)
+static __global__ void __launch_bounds__(kThreads)
 k_copy_elems(uint32_t *__restrict__ dst, const uint32_t *__restrict__ src, uint64_t n) {
     const uint64_t nvec = n >> 2;
     const uint64_t stride = (uint64_t)gridDim.x * kThreads;

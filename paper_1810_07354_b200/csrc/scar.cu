@@ -694,6 +694,7 @@ const char *scar_strerror(int code) {
         case SCAR_ERR_CUDA: return "CUDA runtime error";
         case SCAR_ERR_STATE: return "call not valid in this state";
         case SCAR_ERR_TIMEOUT: return "device-side wait timed out";
+        case SCAR_ERR_CAPACITY: return "problem exceeds a fixed-size internal buffer";
         default: return "unknown error";
     }
 }

@@ -1,0 +1,143 @@
+// scar_perturbation_norm_static: the read-only perturbation norm for callers
+// that must not allocate.
+//
+// Who needs this: code that runs where device allocation is off limits or
+// unaffordable - a failure handler that has to size up the damage while the
+// process is already short of memory, a step of a latency-critical loop where a
+// cudaMalloc (which synchronises the device) is not acceptable, or a host
+// framework that hands a plug-in a fixed memory budget and forbids it to grow.
+// Such callers cannot create a scar_ctx, because scar_ckpt_init allocates the
+// checkpoint copy and its work arrays.
+//
+// The regular norm pass keeps one partial sum per block plus a few per-tile
+// sums and a ticket counter in memory that the context allocated.  Here that
+// scratch is a fixed array in the library's device image instead, so every GPU
+// that loads the library carries it (about 8 MiB) until the process exits, and
+// the block count is capped at SCAR_STATIC_MAX_BLOCKS.
+#include <cstdint>
+#include <mutex>
+
+#include "scar.h"
+
+#include "block_pass.cuh"
+
+using namespace scar;
+
+namespace {
+
+constexpr uint64_t kStaticMaxBlocks = SCAR_STATIC_MAX_BLOCKS;
+constexpr uint64_t kStaticMaxTiles = (kStaticMaxBlocks + kReduceTile - 1) / kReduceTile;
+// 8-byte words: one partial per block, four per-tile arrays, one word for the ticket.
+constexpr uint64_t kPartWords = kStaticMaxBlocks;
+constexpr uint64_t kTileWords = kStaticMaxTiles;
+constexpr uint64_t kScratchWords = kPartWords + 4 * kTileWords + 32;
+
+// In host code this name is only a handle for cudaGetSymbolAddress: it is not
+// a device address and must never be passed to a kernel as one.
+static __device__ __align__(256) unsigned long long g_static_scratch[kScratchWords];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_mu;
+unsigned long long *g_scratch_addr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device, looked up once
+// per device (with that device current) and remembered.
+int scratch_on_current_device(unsigned long long **out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SCAR_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return SCAR_ERR_STATE;
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_scratch_addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return SCAR_ERR_CUDA;
+        }
+        g_scratch_addr[dev] = static_cast<unsigned long long *>(p);
+    }
+    *out = g_scratch_addr[dev];
+    return SCAR_OK;
+}
+
+static_assert(sizeof(NormInfoDev) == sizeof(scar_norm_info), "result layouts must agree");
+
+template <typename T>
+int run_static(const void *d_x, const void *d_z, const Geom &g, const LostSet &S, unsigned long long *scratch,
+               scar_norm_info *d_out, cudaStream_t stream) {
+    using Sc = typename Elem<T>::score_t;
+    Sc *part = reinterpret_cast<Sc *>(scratch);
+    double *tile_sum = reinterpret_cast<double *>(scratch + kPartWords);
+    unsigned long long *tile_l1 = scratch + kPartWords + kTileWords;
+    unsigned long long *tile_blocks = scratch + kPartWords + 2 * kTileWords;
+    unsigned long long *tile_elems = scratch + kPartWords + 3 * kTileWords;
+    unsigned *ticket = reinterpret_cast<unsigned *>(scratch + kPartWords + 4 * kTileWords);
+    // The array keeps whatever the previous call left; only the ticket has to start at zero
+    // (every partial that is read is written first by this call).
+    if (cudaMemsetAsync(ticket, 0, sizeof(unsigned), stream) != cudaSuccess) return SCAR_ERR_CUDA;
+
+    double units = (double)g.n_elems / (double)g.n_blocks;
+    if (g.vec_ok) units /= 4.0;
+    int G = 4;
+    while (G < 32 && G * 4 < units) G <<= 1;
+    const unsigned grid = (unsigned)((g.n_blocks + (kThreads / G) - 1) / (kThreads / G));
+    T *x = static_cast<T *>(const_cast<void *>(d_x));  // the read-only instantiation never stores
+    const T *z = static_cast<const T *>(d_z);
+#define SCAR_STATIC_LAUNCH(G_, VEC_) \
+    k_recover_blocks<T, G_, VEC_, false><<<grid, kThreads, 0, stream>>>(x, z, g, S, part)
+    if (g.vec_ok) {
+        if (G == 4) SCAR_STATIC_LAUNCH(4, true);
+        else if (G == 8) SCAR_STATIC_LAUNCH(8, true);
+        else if (G == 16) SCAR_STATIC_LAUNCH(16, true);
+        else SCAR_STATIC_LAUNCH(32, true);
+    } else {
+        if (G == 4) SCAR_STATIC_LAUNCH(4, false);
+        else if (G == 8) SCAR_STATIC_LAUNCH(8, false);
+        else if (G == 16) SCAR_STATIC_LAUNCH(16, false);
+        else SCAR_STATIC_LAUNCH(32, false);
+    }
+#undef SCAR_STATIC_LAUNCH
+    const unsigned tiles = (unsigned)((g.n_blocks + kReduceTile - 1) / kReduceTile);
+    k_reduce_partials<T><<<tiles, kThreads, 0, stream>>>(part, g, S, tile_sum, tile_l1, tile_blocks, tile_elems, ticket,
+                                                        reinterpret_cast<NormInfoDev *>(d_out));
+    return cudaGetLastError() == cudaSuccess ? SCAR_OK : SCAR_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" int scar_perturbation_norm_static(const void *d_x, const void *d_z, scar_dtype dt, const scar_layout *layout,
+                                             const uint8_t *d_lost_blocks, scar_norm_info *d_out, void *cuda_stream) {
+    if (!layout || !d_out || (dt != SCAR_F32 && dt != SCAR_I32)) return SCAR_ERR_INVALID_ARG;
+    if (layout->block_offsets) return SCAR_ERR_INVALID_ARG;  // explicit offsets would have to be copied to the device
+    if (layout->n_elems > 0 && (!d_x || !d_z)) return SCAR_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_z)) & 15) return SCAR_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (layout->n_elems == 0)
+        return cudaMemsetAsync(d_out, 0, sizeof(scar_norm_info), stream) == cudaSuccess ? SCAR_OK : SCAR_ERR_CUDA;
+    if (layout->block_elems == 0) return SCAR_ERR_LAYOUT;
+    const uint64_t row = layout->row_elems ? layout->row_elems : layout->n_elems;
+    if (row > layout->n_elems || layout->n_elems % row != 0) return SCAR_ERR_LAYOUT;
+    const uint64_t per_row = (row + layout->block_elems - 1) / layout->block_elems;
+    const uint64_t rows = layout->n_elems / row;
+    if (per_row > kStaticMaxBlocks || rows > kStaticMaxBlocks || per_row * rows > kStaticMaxBlocks)
+        return SCAR_ERR_CAPACITY;
+
+    Geom g{};
+    g.n_elems = layout->n_elems;
+    g.row_len = row;
+    g.n_blocks = per_row * rows;
+    g.boff = nullptr;
+    g.block_elems = layout->block_elems;
+    g.blocks_per_row = (uint32_t)per_row;
+    g.n_shards = 1;
+    g.vec_ok = (row % 4 == 0) && (layout->block_elems % 4 == 0);
+    LostSet S{};
+    S.mode = d_lost_blocks ? 2 : 0;
+    S.mask = d_lost_blocks;
+    S.n_work = g.n_blocks;
+
+    unsigned long long *scratch = nullptr;
+    int rc = scratch_on_current_device(&scratch);
+    if (rc != SCAR_OK) return rc;
+    return dt == SCAR_F32 ? run_static<float>(d_x, d_z, g, S, scratch, d_out, stream)
+                          : run_static<int>(d_x, d_z, g, S, scratch, d_out, stream);
+}

@@ -1,0 +1,97 @@
+"""scar_perturbation_norm_static: the perturbation norm for callers that cannot allocate.
+
+A recovery handler that runs when device memory is exhausted, or a plug-in whose host framework
+forbids cudaMalloc, cannot create a context (scar_ckpt_init allocates the checkpoint copy and its
+work arrays).  The static entry point keeps its scratch in a fixed array inside the library, so
+these tests check that it gives exactly what the context-based call gives, twice in a row through
+the shared scratch, that it refuses layouts beyond its fixed capacity, and that device memory in
+use does not grow across a call.  This file sorts last on purpose: a failure here cannot hide the
+results of the other GPU tests.
+"""
+
+import ctypes as C
+
+import numpy as np
+import pytest
+
+from workloads import make_workload
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from paper_1810_07354_b200 import api  # noqa: E402
+
+
+def read_info(d_out: "torch.Tensor") -> api.scar_norm_info:
+    raw = d_out.cpu().numpy().tobytes()
+    return api.scar_norm_info.from_buffer_copy(raw)
+
+
+def reference(x, z, geom, mask_dev, dtype_is_float):
+    """The existing context-based entry point on the same data."""
+    xd = x.clone()
+    ck = api.ScarCheckpoint(xd, n_shards=1, row_elems=geom.row_elems, block_elems=geom.block_elems)
+    ck.load(z)
+    out = ck.perturbation_norm_blocks(mask_dev)
+    ck.close()
+    return out
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", dict(n_elems=1 << 20)), ("mf", dict(l_rows=30_000, r_rows=1_000)),
+                                      ("lda", dict(vocab=3_000, topics=1000))])
+def test_static_norm_matches_context_norm_on_two_calls_in_a_row(name, kw):
+    w = make_workload(name, **kw)
+    is_float = w.x.dtype == np.float32
+    dt = api.SCAR_F32 if is_float else api.SCAR_I32
+    x = torch.from_numpy(w.x).cuda()
+    z = torch.from_numpy(w.z).cuda()
+    nb = w.n_blocks
+    rng = np.random.Generator(np.random.PCG64(99))
+    masks = [torch.from_numpy((rng.random(nb) < 0.3).astype(np.uint8)).cuda(), None,
+             torch.from_numpy((rng.random(nb) < 0.7).astype(np.uint8)).cuda()]
+    want = [reference(x, z, w.geom, m, is_float) for m in masks]
+    layout = api.make_layout(w.x.size, w.geom.row_elems, w.geom.block_elems, 1)
+    d_out = torch.zeros(4, dtype=torch.int64, device="cuda")  # 32 bytes = one scar_norm_info
+    stream = torch.cuda.current_stream().cuda_stream
+    # first call (does the one-time address look-up), then measure memory around the next ones
+    api.scar_perturbation_norm_static(x, z, dt, layout, masks[0], d_out, stream)
+    torch.cuda.synchronize()
+    got0 = read_info(d_out)
+    free_before = torch.cuda.mem_get_info()[0]
+    got = [got0]
+    for m in masks[1:]:
+        api.scar_perturbation_norm_static(x, z, dt, layout, m, d_out, stream)
+        torch.cuda.synchronize()
+        got.append(read_info(d_out))
+    assert torch.cuda.mem_get_info()[0] == free_before, "the call must not change device memory in use"
+    for g, wnt in zip(got, want):
+        assert (g.lost_blocks, g.lost_elems, g.l1) == (wnt.lost_blocks, wnt.lost_elems, wnt.l1)
+        if is_float:
+            assert abs(g.l2 - wnt.l2) <= 1e-5 * wnt.l2
+            assert g.l2 == wnt.l2, "same kernels, same order of additions: identical bits expected"
+        else:
+            assert g.l2 == 0.0
+    # inputs are read-only
+    assert x.cpu().numpy().tobytes() == w.x.tobytes() and z.cpu().numpy().tobytes() == w.z.tobytes()
+
+
+def test_static_norm_rejects_what_it_cannot_hold():
+    lib = api.load_library()
+    d_out = torch.zeros(4, dtype=torch.int64, device="cuda")
+    buf = torch.zeros(1 << 12, dtype=torch.float32, device="cuda")
+    too_many = api.make_layout((1 << 20) + 1, 0, 1, 1)  # one block more than SCAR_STATIC_MAX_BLOCKS
+    rc = lib.scar_perturbation_norm_static(buf.data_ptr(), buf.data_ptr(), 0, C.byref(too_many), None,
+                                           d_out.data_ptr(), None)
+    assert rc == -7 and "fixed-size" in api.scar_strerror(rc)
+    explicit = api.make_layout(8, block_offsets=np.array([0, 4, 8], dtype=np.uint64))
+    assert lib.scar_perturbation_norm_static(buf.data_ptr(), buf.data_ptr(), 0, C.byref(explicit), None,
+                                             d_out.data_ptr(), None) == -1
+    ok = api.make_layout(1 << 12, 0, 256, 1)
+    assert lib.scar_perturbation_norm_static(buf.data_ptr() + 4, buf.data_ptr(), 0, C.byref(ok), None,
+                                             d_out.data_ptr(), None) == -1, "misaligned x"
+    assert lib.scar_perturbation_norm_static(buf.data_ptr(), buf.data_ptr(), 0, C.byref(ok), None, None, None) == -1
+    # a valid call right after the refusals still works: x == z gives a zero perturbation
+    api.scar_perturbation_norm_static(buf, buf, api.SCAR_F32, ok, None, d_out)
+    torch.cuda.synchronize()
+    info = read_info(d_out)
+    assert info.l2 == 0.0 and info.lost_blocks == 16 and info.lost_elems == 1 << 12
