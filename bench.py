@@ -1,21 +1,22 @@
 #!/usr/bin/env python
-"""Benchmark of the SCAR checkpoint-and-recover pass on the CNN-scale parameter set.
+"""Benchmark of the SCAR checkpoint-and-recover pass.
 
-One step = the whole hot path over one synthetic parameter set of 2**30 float32 elements in
-4096-element blocks: a prioritized save at every r of the sweep (0.01, 0.1, 0.5, 1.0; the running
-checkpoint is put back to its pristine state before each, outside the timed region), the read-only
-full-recovery perturbation norm, and a partial recovery of one of eight shards.  Every timed call is
-bracketed by CUDA events on the stream the library launches on; a step's time is the sum of its
-timed calls.
+Default workload: the CNN-scale parameter set, 2**30 float32 elements in 4096-element blocks.  One
+step = the whole hot path over one synthetic parameter set: a prioritized save at every r of the set's
+sweep (CNN: 0.01, 0.1, 0.5, 1.0; the running checkpoint is put back to its pristine state and L2 is
+flushed before each, outside the timed intervals), the read-only full-recovery perturbation norm, and
+a partial recovery of the set's lost shards or blocks.  Every timed call is bracketed by CUDA events on
+the stream the library launches on; a step's time is the sum of its timed calls.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
 
-With N > 1 (launched by torch.distributed.run) every rank runs an independent replica on its own
-GPU: the method's pass over one device's parameters needs no exchange, so there is no collective on
-the data path; the reported value is the sum over ranks divided by the slowest rank's time.
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica on its own GPU:
+the pass over one device's parameters needs no exchange, so there is no collective on the data path;
+the reported value is the sum over ranks divided by the slowest rank's time.
 
-``--impl reference`` times the plain CPU oracle (``oracle/``) on the host cores over a bounded
-sample of the same parameter set, with the same metric.
+``--impl reference`` times the plain CPU oracle (``oracle/``) on the host cores over a bounded sample
+of the same parameter set, with the same metric.  ``--workload`` selects one of the other synthetic
+sets (tiny, mlr, mf, lda) for the same measurement.
 """
 
 from __future__ import annotations
@@ -26,7 +27,6 @@ import os
 import subprocess
 import sys
 import tempfile
-import threading
 import time
 
 import numpy as np
@@ -35,13 +35,24 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-R_SWEEP = (0.01, 0.1, 0.5, 1.0)
 N_ELEMS = 1 << 30
 BLOCK = 4096
 ELEM = 4
 METRIC = "prioritized-checkpoint GB/s scanned"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
+
+DESCRIPTIONS = {
+    "cnn": "cnn-scale fp32 vector, block 4096, r sweep 0.01/0.1/0.5/1.0 + full norm + recovery of 1 of 8 shards",
+    "mlr": "mlr-shaped fp32 1000x100000, blocks of 1024 within rows, r 0.05/0.25 + full norm + recovery of 1 of 8 "
+           "row shards",
+    "mf": "mf-shaped fp32 factors (480000+18000)x100, one 100-float row per block, r 0.1 + full norm + recovery of "
+          "a random 25% of L rows",
+    "lda": "lda-shaped int32 100000x1000 count table, one row per block, integer l1, r 0.2 + full norm + recovery "
+           "of 2 of 8 shards",
+    "tiny": "tiny fp32 vector 2**20, block 256, r 0.25 + full norm + recovery of 4 of 8 shards (L2-resident: "
+            "latency-bound, not an HBM measurement)",
+}
 
 
 def hbm_peak():
@@ -53,15 +64,15 @@ def hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def recorded_traffic(n_elems: int):
-    """DRAM bytes per k_block_scores launch from the last ncu capture, scaled to n_elems; None when there
-    is no capture or the kernel sources changed after it was taken."""
+def recorded_traffic(n_elems: int, kernel: str = "k_block_scores"):
+    """DRAM bytes per launch of the dominant kernel from the last ncu capture, scaled to n_elems; None when
+    there is no capture or the kernel sources changed after it was taken."""
     import hashlib
 
     pkg = os.path.join(ROOT, "paper_1810_07354_b200")
     try:
         with open(os.path.join(pkg, "ncu_traffic.json")) as f:
-            rec = json.load(f)["k_block_scores"]
+            rec = json.load(f)[kernel]
         h = hashlib.sha256()
         for name in ("geom.cuh", "block_pass.cuh"):
             with open(os.path.join(pkg, "csrc", name), "rb") as f:
@@ -136,56 +147,69 @@ class ClockSampler:
 # ----------------------------------------------------------------------------- CPU oracle legs
 
 
-def oracle_step(x, z, boff, lost_blocks, timers):
+def oracle_step(x, z, boff, lost_blocks, r_sweep):
     """One step of the hot path on the oracle; returns seconds spent in saves and in total."""
     import oracle
 
     t_save = 0.0
     t0 = time.perf_counter()
-    for r in R_SWEEP:
+    for r in r_sweep:
         t = time.perf_counter()
         oracle.priority_save(x, z, boff, r=r)
         t_save += time.perf_counter() - t
-    t = time.perf_counter()
     oracle.perturbation_norm(x, z, boff, None)
     oracle.recover_partial(x, z, boff, lost_blocks)
-    timers["recover_s"] = timers.get("recover_s", 0.0) + time.perf_counter() - t
     return t_save, time.perf_counter() - t0
 
 
+def host_workload(name: str, n_elems: int):
+    """Host (numpy) form of a workload; only the CNN-scale set takes a size."""
+    from workloads import make_workload
+
+    if name == "cnn":
+        return make_workload("cnn", n_elems=n_elems, block_elems=BLOCK)
+    return make_workload(name)
+
+
+def lost_block_mask(w):
+    import oracle
+
+    return w.lost_blocks if w.lost_blocks is not None else oracle.expand_shards(w.n_blocks, w.lost_shards)
+
+
 def run_reference(args):
-    """The oracle as it stands, single-threaded, on a bounded sample of the CNN-scale set."""
+    """The oracle as it stands, single-threaded, on a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import oracle
-    from workloads import block_offsets, make_workload
+    from workloads import block_offsets
 
-    # One oracle step over 2**26 elements takes about 5 s; shrink the sample so that warm-up plus
-    # timed steps stay within a couple of minutes.
+    # One oracle step over 2**26 CNN-scale elements takes 2-5 s; shrink the sample so that warm-up plus
+    # timed steps stay within a couple of minutes.  The other sets (<= 1e8 elements) are used whole.
     n = 1 << 26
     while n > (1 << 22) and 5.0 * (n / (1 << 26)) * (args.steps + args.warmup) > 120.0:
         n >>= 1
     n = max(BLOCK, min(n, args.n_elems))
-    w = make_workload("cnn", n_elems=n, block_elems=BLOCK)
+    w = host_workload(args.workload, n)
+    n = w.x.size
+    full = N_ELEMS if args.workload == "cnn" else n
     boff = block_offsets(w.geom)
-    lost = oracle.expand_shards(w.n_blocks, w.lost_shards)
-    timers = {}
+    lost = lost_block_mask(w)
     for _ in range(args.warmup):
-        oracle_step(w.x, w.z, boff, lost, timers)
+        oracle_step(w.x, w.z, boff, lost, w.r_values)
     t_save = t_all = 0.0
     for _ in range(args.steps):
-        a, b = oracle_step(w.x, w.z, boff, lost, timers)
+        a, b = oracle_step(w.x, w.z, boff, lost, w.r_values)
         t_save += a
         t_all += b
-    value = len(R_SWEEP) * 2 * n * ELEM * args.steps / t_save / 1e9
-    sample = f"first {n} of {N_ELEMS} elements ({w.n_blocks} blocks), numpy-generated with the same recipe"
+    value = len(w.r_values) * 2 * n * ELEM * args.steps / t_save / 1e9
+    sample = f"{n} of {full} elements ({w.n_blocks} blocks), numpy-generated with the same recipe"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_all / args.steps,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "cnn-scale fp32 vector, block 4096, r sweep 0.01/0.1/0.5/1.0 + full norm + "
-                               "recovery of 1 of 8 shards", "n_elems": n, "sample_of": N_ELEMS},
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64" if w.dtype == "f32" else "int64", "data": "synthetic",
+        "config": {"workload": DESCRIPTIONS[args.workload], "n_elems": n, "sample_of": full},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -193,19 +217,20 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def cpu_baseline(x_dev, z_dev, lost_shards):
-    """Times the oracle on a prefix of the device-resident workload (copied to the host)."""
-    import oracle
+def cpu_baseline(x_dev, z_dev, geom, lost_blocks, r_sweep):
+    """Times one oracle step on the device-resident workload (copied to the host), single thread."""
+    from workloads import block_offsets
 
-    n = min(x_dev.numel(), 1 << 30)
-    nb = n // BLOCK
-    x = x_dev[:n].cpu().numpy()
-    z = z_dev[:n].cpu().numpy()
-    boff = oracle.layout_offsets(n, 0, BLOCK)
-    lost = oracle.expand_shards(nb, lost_shards)
-    t_save, _ = oracle_step(x, z, boff, lost, {})
-    return {"value": len(R_SWEEP) * 2 * n * ELEM / t_save / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"one step on {n} of {N_ELEMS} elements ({nb} blocks) of the same buffers, "
+    x = x_dev.cpu().numpy()
+    z = z_dev.cpu().numpy()
+    boff = block_offsets(geom)
+    reps, t_save = 0, 0.0
+    while reps < 1 or (t_save < 5.0 and reps < 50):  # small sets: repeat until a few seconds have been timed
+        t_save += oracle_step(x, z, boff, lost_blocks, r_sweep)[0]
+        reps += 1
+    return {"value": reps * len(r_sweep) * 2 * x.size * ELEM / t_save / 1e9, "unit": UNIT, "cores": 1,
+            "kind": "oracle",
+            "sample": f"{reps} step(s) on all {x.size} elements ({geom.n_blocks} blocks) of the same buffers, "
                       f"single thread, {t_save:.1f} s in saves"}
 
 
@@ -229,12 +254,27 @@ def job_throughput_gbs(world, bytes_per_rank, max_ms):
     return world * bytes_per_rank / (max_ms * 1e-3) / 1e9
 
 
+def device_workload(name, n_elems, rank, dev):
+    """(geom, z0, x0, r_sweep, lost_shards, lost_blocks_host) with z0 / x0 on the device."""
+    import torch
+
+    if name == "cnn":
+        from workloads.configs import make_cnn_device
+
+        geom, z0, x0, lost_shards = make_cnn_device(n_elems, BLOCK, seed=4 + rank, device=dev)
+        return geom, z0, x0, (0.01, 0.1, 0.5, 1.0), lost_shards, None
+    from workloads import make_workload
+
+    w = make_workload(name)
+    return (w.geom, torch.from_numpy(w.z).to(dev), torch.from_numpy(w.x).to(dev), w.r_values, w.lost_shards,
+            w.lost_blocks)
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
 
     from paper_1810_07354_b200 import api
-    from workloads.configs import make_cnn_device
 
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback for the library")
@@ -252,15 +292,18 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    n = args.n_elems
-    geom, z0, x0, lost_shards = make_cnn_device(n, BLOCK, seed=4 + rank, device=dev)
+    geom, z0, x0, r_sweep, lost_shards, lost_blocks = device_workload(args.workload, args.n_elems, rank, dev)
+    n = x0.numel()
     x = x0.clone()
-    ck = api.ScarCheckpoint(x, n_shards=8, block_elems=BLOCK)
+    ck = api.ScarCheckpoint(x, n_shards=geom.n_shards, row_elems=geom.row_elems, block_elems=geom.block_elems)
     ctx = ck.ctx
     nb = ck.n_blocks
-    shard_lo = int(np.flatnonzero(lost_shards)[0]) * (nb // 8) * BLOCK
-    shard_hi = shard_lo + (nb // 8) * BLOCK
-    lost_elems = shard_hi - shard_lo
+    d_lost = torch.from_numpy(lost_blocks).to(dev) if lost_blocks is not None else None
+
+    def recover(sync=False):
+        if d_lost is not None:
+            return ck.recover_partial_blocks(d_lost, sync=sync)
+        return ck.recover_partial(lost_shards, sync=sync)
 
     z_lib = ck.views()["z"]  # the library's running checkpoint, aliased (no copy)
     flush = torch.empty(64 << 20, dtype=torch.float32, device=dev)  # 256 MiB, larger than the 126 MB L2
@@ -270,29 +313,37 @@ def run_gpu(args):
         z_lib.copy_(z0)
         flush.zero_()
 
+    def reset_live():
+        x.copy_(x0)
+        flush.zero_()
+
+    lost_elems = int(recover(sync=True).lost_elems)
+    reset_live()
+
     ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
 
     def one_step(rec):
         """Runs one step; appends (kind, start_event, end_event) triples to rec."""
-        for r in R_SWEEP:
+        for r in r_sweep:
             reset_checkpoint()
             a, b = ev(), ev()
             a.record()
             ck.priority_save(r, sync=False)
             b.record()
             rec.append((("save", r), a, b))
+        reset_checkpoint()
         a, b = ev(), ev()
         a.record()
         ck.perturbation_norm(None, sync=False)
         b.record()
         rec.append((("norm", None), a, b))
+        flush.zero_()
         a, b = ev(), ev()
         a.record()
-        ck.recover_partial(lost_shards, sync=False)
+        recover()
         b.record()
         rec.append((("recover", None), a, b))
-        x[shard_lo:shard_hi].copy_(x0[shard_lo:shard_hi])  # put the live parameters back (not timed)
-        flush.zero_()
+        reset_live()  # put the live parameters back (not timed)
 
     for _ in range(args.warmup):
         one_step([])
@@ -300,7 +351,7 @@ def run_gpu(args):
 
     # payload sizes per r (data dependent but fixed for this workload)
     payload_elems = {}
-    for r in R_SWEEP:
+    for r in r_sweep:
         reset_checkpoint()
         payload_elems[r] = int(ck.priority_save(r).payload_elems)
     barrier()
@@ -327,18 +378,19 @@ def run_gpu(args):
 
     # ---- dominant kernel (block scores) timed live through the library's own stream events
     api.scar_ckpt_profile(ctx, True)
-    phase = {r: [] for r in R_SWEEP}
+    phase = {r: [] for r in r_sweep}
     rec_phase = []
     for _ in range(min(args.steps, 10)):
-        for r in R_SWEEP:
+        for r in r_sweep:
             reset_checkpoint()
             ck.priority_save(r, sync=False)
             phase[r].append(api.scar_ckpt_profile_read(ctx))
-        ck.recover_partial(lost_shards, sync=False)
+        flush.zero_()
+        recover()
         rec_phase.append(api.scar_ckpt_profile_read(ctx))
-        x[shard_lo:shard_hi].copy_(x0[shard_lo:shard_hi])
+        reset_live()
     api.scar_ckpt_profile(ctx, False)
-    score_ms = float(np.mean([p[0] for r in R_SWEEP for p in phase[r]]))
+    score_ms = float(np.mean([p[0] for r in r_sweep for p in phase[r]]))
 
     if rank != 0:
         barrier()
@@ -348,9 +400,9 @@ def run_gpu(args):
 
     peak, peak_kind = hbm_peak()
     scanned = 2 * n * ELEM
-    value = job_throughput_gbs(world, len(R_SWEEP) * scanned * args.steps, save_ms)
+    value = job_throughput_gbs(world, len(r_sweep) * scanned * args.steps, save_ms)
     per_r = {}
-    for r in R_SWEEP:
+    for r in r_sweep:
         ms = float(np.median(t[("save", r)]))
         by = save_bytes(n, payload_elems[r])
         ph = np.median(np.array(phase[r]), axis=0)
@@ -362,16 +414,15 @@ def run_gpu(args):
     rec_ms = float(np.median(t[("recover", None)]))
     rph = np.median(np.array(rec_phase), axis=0)
     achieved = scanned / (score_ms * 1e-3) / 1e9
+    l2_note = ("inputs larger than L2; " if scanned > (512 << 20) else "inputs NOT larger than L2; ") + \
+        "L2 flushed by a 256 MiB write after every untimed state reset and before every timed call"
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": tot_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "cnn-scale fp32 vector, block 4096, r sweep 0.01/0.1/0.5/1.0 + full norm + "
-                               "recovery of 1 of 8 shards", "n_elems": n, "n_blocks": nb, "r_sweep": list(R_SWEEP),
-                   "l2": "inputs larger than L2 (8 GiB scanned per save); L2 also flushed by a 256 MiB write "
-                         "after every untimed state reset",
-                   "value_is": "sum over the r sweep of 2*N*4 bytes / sum of save times",
+        "dtype": "f32" if x0.dtype == torch.float32 else "int32", "data": "synthetic",
+        "config": {"workload": DESCRIPTIONS[args.workload], "n_elems": n, "n_blocks": nb, "r_sweep": list(r_sweep),
+                   "l2": l2_note, "value_is": "sum over the r sweep of 2*N*4 bytes / sum of save times",
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
         "save_ms_per_step": save_ms / args.steps,
         "per_r": per_r,
@@ -379,7 +430,8 @@ def run_gpu(args):
         "partial_recovery": {"ms": rec_ms, "gbs": 3 * lost_elems * ELEM / rec_ms / 1e6, "lost_elems": lost_elems,
                              "phase_ms": {"restore": float(rph[3]), "reduce": float(rph[4])}},
         "roofline": {"bound": "hbm", "kernel": "k_block_scores", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": recorded_traffic(n),
+                     "frac": achieved / peak, "peak_source": f"of {peak_kind}",
+                     "traffic": recorded_traffic(n) if args.workload == "cnn" else None,
                      "bytes_per_launch": scanned, "ms_per_launch": score_ms},
         "gpu_launches": int(launches),
         "clocks": clocks,
@@ -387,23 +439,32 @@ def run_gpu(args):
     }
 
     if not args.no_e2e:
-        line["e2e"] = run_e2e(api, ck, x, x0, z0, lost_shards, shard_lo, shard_hi, n, nb, world)
+        line["e2e"] = run_e2e(api, ck, x0, z_lib, z0, r_sweep, lost_shards, lost_elems, n, nb, world, flush)
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(x0, z0, lost_shards)
+        if lost_blocks is None:
+            from workloads import shard_block_ranges
+
+            lb = np.zeros(nb, dtype=np.uint8)
+            for lo, hi in shard_block_ranges(nb, geom.n_shards)[np.flatnonzero(lost_shards)]:
+                lb[lo:hi] = 1
+        else:
+            lb = lost_blocks
+        line["cpu_baseline"] = cpu_baseline(x0, z0, geom, lb, r_sweep)
     print(json.dumps(line))
     barrier()
     if world > 1:
         dist.destroy_process_group()
 
 
-def run_e2e(api, ck, x, x0, z0, lost_shards, shard_lo, shard_hi, n, nb, world):
+def run_e2e(api, ck, x0, z_lib, z0, r_sweep, lost_shards, lost_elems, n, nb, world, flush):
     """Same step through the host-buffer entry points: every save uploads x from pinned host memory and
-    downloads ids, offsets and payload; the recovery uploads and downloads the lost shard."""
+    downloads ids, offsets and payload; the recovery (shard-mask workloads) uploads and downloads the lost
+    shards.  Wall-clock around the synchronous calls, copies included."""
     import torch
 
-    hx = torch.empty(n, dtype=torch.float32).pin_memory()
+    hx = torch.empty(n, dtype=x0.dtype).pin_memory()
     hx.copy_(x0)
-    h_payload = torch.empty(n, dtype=torch.float32).pin_memory()
+    h_payload = torch.empty(n, dtype=x0.dtype).pin_memory()
     h_sel = torch.empty(nb, dtype=torch.int32).pin_memory()
     h_poff = torch.empty(nb + 1, dtype=torch.int64).pin_memory()
     steps = 2
@@ -411,26 +472,30 @@ def run_e2e(api, ck, x, x0, z0, lost_shards, shard_lo, shard_hi, n, nb, world):
     h2d = d2h = 0
     for it in range(steps + 1):
         torch.cuda.synchronize()
-        s0 = time.perf_counter()
+        t_step = 0.0
         ts = 0.0
         h2d = d2h = 0
-        for r in R_SWEEP:
-            ck.load(z0)  # untimed reset
+        for r in r_sweep:
+            z_lib.copy_(z0)  # untimed reset
+            flush.zero_()
             torch.cuda.synchronize()
             a = time.perf_counter()
             info = api.scar_ckpt_priority_save_host(ck.ctx, hx, r, h_payload, h_sel, h_poff)
             ts += time.perf_counter() - a
             h2d += n * ELEM
             d2h += int(info.payload_elems) * ELEM + int(info.k) * 4 + (int(info.k) + 1) * 8 + 24
-        api.scar_recover_partial_host(ck.ctx, hx, lost_shards)
-        h2d += (shard_hi - shard_lo) * ELEM + 8
-        d2h += (shard_hi - shard_lo) * ELEM + 32
-        torch.cuda.synchronize()
+        t_step += ts
+        if lost_shards is not None:
+            a = time.perf_counter()
+            api.scar_recover_partial_host(ck.ctx, hx, lost_shards)
+            t_step += time.perf_counter() - a
+            h2d += lost_elems * ELEM
+            d2h += lost_elems * ELEM + 32
+            hx.copy_(x0)
         if it > 0:  # first pass is a warm-up
             t_save += ts
-            t_all += time.perf_counter() - s0
-        hx[shard_lo:shard_hi].copy_(x0[shard_lo:shard_hi])
-    return {"value": world * len(R_SWEEP) * 2 * n * ELEM * steps / t_save / 1e9, "unit": UNIT,
+            t_all += t_step
+    return {"value": world * len(r_sweep) * 2 * n * ELEM * steps / t_save / 1e9, "unit": UNIT,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * t_all / steps,
             "note": "host-buffer C-ABI calls, pinned host memory, copies inside the timed region"}
 
@@ -441,7 +506,9 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--n-elems", type=int, default=N_ELEMS, help="elements of the parameter vector (default 2**30)")
+    ap.add_argument("--workload", default="cnn", choices=sorted(DESCRIPTIONS))
+    ap.add_argument("--n-elems", type=int, default=N_ELEMS,
+                    help="elements of the CNN-scale parameter vector (default 2**30)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

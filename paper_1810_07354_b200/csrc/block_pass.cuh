@@ -46,8 +46,7 @@ template <> struct Elem<int> {
     using score_t = unsigned long long;
     using acc_t = unsigned long long;
     static __device__ __forceinline__ void add(acc_t &a, int x, int z) {
-        unsigned d = x > z ? (unsigned)x - (unsigned)z : (unsigned)z - (unsigned)x;
-        a += d;
+        a += __sad(x, z, 0u);  // |x - z| as an unsigned 32-bit value, exact for any pair of int32
     }
     static __device__ __forceinline__ void addu(acc_t &a, int x, int z) { add(a, x, z); }
     static __device__ __forceinline__ void addu(acc_t &a, const vec_t &x, const vec_t &z) {
@@ -115,8 +114,10 @@ __device__ __forceinline__ typename Elem<T>::wide_t block_distance(T *__restrict
     unsigned it = 0;
     if (!WRITE) {
         // Read-only pass: nothing can hold back the loads, so the plain loop is
-        // the faster form (full batches unguarded, then one guarded batch).
-        for (; u + 3 * (uint64_t)G < n; u += step) {
+        // the faster form (full batches unguarded, then one guarded batch).  A
+        // batch counts as full only when it is full for every lane of the group,
+        // so the lanes of a group never diverge between the two forms.
+        for (; u - lane + step <= n; u += step) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 xc[j] = ld_stream(xs + u + (uint64_t)j * G);
@@ -203,6 +204,30 @@ k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S,
                  typename Elem<T>::score_t *__restrict__ part) {
     using E = Elem<T>;
     const int lane = threadIdx.x & (G - 1);
+    if (G < 32 && S.mode == 2) {
+        // Per-block mask with several blocks per warp: a warp takes 32 consecutive
+        // blocks, ballots which are lost and hands only those to its groups, so that
+        // a sparse mask does not leave most lanes idle.
+        constexpr int kGroups = 32 / G;
+        const int wl = threadIdx.x & 31, gi = wl / G;
+        const uint64_t b0 = (((uint64_t)blockIdx.x * kThreads + threadIdx.x) >> 5) * 32;
+        const bool lost = b0 + wl < g.n_blocks && S.mask[b0 + wl] != 0;
+        const unsigned bal = __ballot_sync(0xffffffffu, lost);
+        const int cnt = __popc(bal);
+        for (int t0 = 0; t0 < cnt; t0 += kGroups) {  // same trip count for every lane of the warp
+            const int t = t0 + gi;
+            const bool valid = t < cnt;
+            uint32_t b = 0;
+            uint64_t beg = 0, len = 0;
+            if (valid) {
+                b = (uint32_t)(b0 + __fns(bal, 0, t + 1));
+                g.range(b, beg, len);
+            }
+            typename E::wide_t s = block_distance<T, G, VEC, WRITE>(x, z, beg, len, lane);
+            if (valid && lane == 0) part[b] = (typename E::score_t)s;
+        }
+        return;
+    }
     const uint64_t w = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
     uint32_t b = 0;
     const bool valid = S.block_of(w, b);

@@ -220,7 +220,9 @@ template <typename T> void launch_recover(scar_ctx *c, const LostSet &S, bool wr
         dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
             constexpr int G = decltype(gl)::value;
             constexpr bool VEC = decltype(vec)::value;
-            const unsigned grid = grid_for_groups(S.n_work, G);
+            // a per-block mask with several blocks per warp is walked 32 blocks per warp
+            const unsigned grid = (G < 32 && S.mode == 2) ? (unsigned)((S.n_work + kThreads - 1) / kThreads)
+                                                          : grid_for_groups(S.n_work, G);
             if (write)
                 k_recover_blocks<T, G, VEC, true><<<grid, kThreads, 0, c->stream>>>(
                     static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, static_cast<Sc *>(c->part));

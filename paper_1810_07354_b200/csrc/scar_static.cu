@@ -79,7 +79,8 @@ int run_static(const void *d_x, const void *d_z, const Geom &g, const LostSet &S
     if (g.vec_ok) units /= 4.0;
     int G = 4;
     while (G < 32 && G * 4 < units) G <<= 1;
-    const unsigned grid = (unsigned)((g.n_blocks + (kThreads / G) - 1) / (kThreads / G));
+    const unsigned grid = (G < 32 && S.mode == 2) ? (unsigned)((g.n_blocks + kThreads - 1) / kThreads)
+                                                  : (unsigned)((g.n_blocks + (kThreads / G) - 1) / (kThreads / G));
     T *x = static_cast<T *>(const_cast<void *>(d_x));  // the read-only instantiation never stores
     const T *z = static_cast<const T *>(d_z);
 #define SCAR_STATIC_LAUNCH(G_, VEC_) \

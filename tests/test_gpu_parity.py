@@ -94,6 +94,35 @@ def test_cnn_reduced_all_r():
     run_save_and_recover(w, w.r_values)
 
 
+def test_cnn_full_size_in_the_benchmark_configuration():
+    """2**30 elements, 262 144 blocks of 4096, 8 shards: the launch configuration bench.py times.
+
+    The parameter set comes from the seeded device generator the benchmark uses; the oracle gets the
+    same bytes through a device-to-host copy and is run in full (about 10 s of CPU time per sweep)."""
+    from workloads.configs import make_cnn_device
+
+    geom, z_dev, x_dev, lost_shards = make_cnn_device(1 << 30, 4096, seed=4, device="cuda:0")
+    x_host, z_host = x_dev.cpu().numpy(), z_dev.cpu().numpy()
+    boff = block_offsets(geom)
+    ck = api.ScarCheckpoint(x_dev, n_shards=8, block_elems=4096)
+    assert ck.n_blocks == 262_144
+    for r, k in zip((0.01, 0.1, 0.5, 1.0), (2621, 26_214, 131_072, 262_144)):
+        ck.load(z_dev)
+        ora = oracle.priority_save(x_host, z_host, boff, r=r)
+        assert ora.k == k
+        info = ck.priority_save(r)
+        parity.check_save(ck, info, x_host, z_host, boff, ora)
+        del ora
+    ck.load(z_dev)
+    parity.check_norm(ck.perturbation_norm(None), oracle.perturbation_norm(x_host, z_host, boff, None), True)
+    lb = oracle.expand_shards(262_144, lost_shards)
+    ora_n, x_after = oracle.recover_partial(x_host, z_host, boff, lb)
+    parity.check_norm(ck.recover_partial(lost_shards), ora_n, True)
+    assert parity.same_bits(x_dev.cpu().numpy(), x_after), "restored buffer differs from the oracle's"
+    assert ora_n.lost_elems == 1 << 27
+    ck.close()
+
+
 # ------------------------------------------------------------------ geometry variants and ragged tails
 
 
