@@ -50,7 +50,8 @@ enum {
     SCAR_ERR_ALLOC = -3,       /* device or host allocation failed */
     SCAR_ERR_CUDA = -4,        /* a CUDA runtime call or kernel launch failed */
     SCAR_ERR_STATE = -5,       /* call not valid in the context's current state */
-    SCAR_ERR_TIMEOUT = -6,     /* reserved: a bounded device-side wait gave up */
+    SCAR_ERR_TIMEOUT = -6,     /* a bounded device-side wait (grid barrier of the selection) gave up;
+                                  the save's outputs are invalid, the context stays usable */
     SCAR_ERR_CAPACITY = -7     /* problem larger than a fixed-size internal buffer */
 };
 

@@ -42,8 +42,9 @@ struct scar_ctx {
     uint8_t *d_shard_mask = nullptr;
     uint8_t *d_block_mask = nullptr;  // only used when a shard mask has too many runs
     SelState *st = nullptr;
-    TileArrays ta{};
+    CtaArrays ca{};
     unsigned n_sel_tiles = 0;
+    unsigned sel_grid = 1, sel_tiles_per_cta = 1;  // launch shape of the cooperative selection kernel
     double *rt_sum = nullptr;
     unsigned long long *rt_l1 = nullptr, *rt_blocks = nullptr, *rt_elems = nullptr;
     unsigned n_red_tiles = 0;
@@ -181,23 +182,31 @@ template <typename T> void launch_scores(scar_ctx *c) {
     ++c->launches;
 }
 
-// a2
-template <typename K, typename S> void launch_select(scar_ctx *c, uint64_t k) {
-    using KT = KeyTraits<K>;
-    const unsigned nt = c->n_sel_tiles;
+// a2: one cooperative launch (all CTAs resident, so its grid-wide barriers cannot deadlock)
+template <typename K, typename S> int launch_select(scar_ctx *c, uint64_t k) {
     const S *score = static_cast<const S *>(c->score);
-    if (k > 0) {
-        for (int p = 0; p < KT::kPasses; ++p) {
-            k_radix_pass<K, S><<<nt, kThreads, 0, c->stream>>>(score, c->g.n_blocks, k, p, c->st);
-            ++c->launches;
-        }
-    }
-    k_select_count<K, S><<<nt, kThreads, 0, c->stream>>>(score, c->g, k, c->st, c->ta, c->d_save, c->poff);
+    unsigned long long kk = k;
+    unsigned nt = c->n_sel_tiles, per = c->sel_tiles_per_cta;
+    void *args[] = {&score, &c->g, &kk, &c->st, &c->ca, &c->d_save, &c->sel, &c->poff, &nt, &per};
+    CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select<K, S>), dim3(c->sel_grid),
+                                       dim3(kThreads), args, 0, c->stream));
     ++c->launches;
-    if (k > 0) {
-        k_select_emit<K, S><<<nt, kThreads, 0, c->stream>>>(score, c->g, c->st, c->ta, c->sel, c->poff);
-        ++c->launches;
-    }
+    return SCAR_OK;
+}
+
+// Grid of the selection kernel: contiguous tile ranges over at most two CTAs per
+// SM (few enough that a barrier costs about a microsecond, and always resident).
+template <typename K, typename S> int plan_select(scar_ctx *c) {
+    int coop = 0, sms = 0, occ = 0;
+    CU_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
+    CU_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device));
+    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_select<K, S>, kThreads, 0));
+    if (!coop || sms < 1 || occ < 1) return SCAR_ERR_CUDA;
+    const unsigned cap = (unsigned)sms * (unsigned)(occ < 2 ? occ : 2);
+    const unsigned nt = c->n_sel_tiles;
+    c->sel_tiles_per_cta = (nt + cap - 1) / cap;
+    c->sel_grid = (nt + c->sel_tiles_per_cta - 1) / c->sel_tiles_per_cta;
+    return SCAR_OK;
 }
 
 // a3
@@ -255,6 +264,12 @@ int copy_elems(scar_ctx *c, void *dst, const void *src, uint64_t n) {
 int fetch_save(scar_ctx *c, scar_save_info *out) {
     CU_TRY(cudaMemcpyAsync(c->h_save, c->d_save, sizeof(SaveInfoDev), cudaMemcpyDeviceToHost, c->stream));
     CU_TRY(cudaStreamSynchronize(c->stream));
+    if (c->h_save->error) {
+        // A grid barrier of the selection gave up; its outputs are not valid.  The kernel has
+        // already put its barrier state back, so the context stays usable.
+        CU_TRY(cudaMemsetAsync(&c->d_save->error, 0, sizeof(unsigned long long), c->stream));
+        return SCAR_ERR_TIMEOUT;
+    }
     out->k = c->h_save->k;
     out->payload_elems = c->h_save->payload_elems;
     out->nonfinite_blocks = c->h_save->nonfinite_blocks;
@@ -294,8 +309,9 @@ int enqueue_save(scar_ctx *c, uint64_t k) {
     if (c->dt == SCAR_F32) launch_scores<float>(c);
     else launch_scores<int>(c);
     record(c, 1);
-    if (c->dt == SCAR_F32) launch_select<unsigned, float>(c, k);
-    else launch_select<unsigned long long, unsigned long long>(c, k);
+    const int rc_sel = c->dt == SCAR_F32 ? launch_select<unsigned, float>(c, k)
+                                         : launch_select<unsigned long long, unsigned long long>(c, k);
+    if (rc_sel != SCAR_OK) return rc_sel;
     c->ran_select = true;
     record(c, 2);
     launch_pack(c, k);
@@ -419,7 +435,7 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     if (c->n_sel_tiles == 0) c->n_sel_tiles = 1;
     c->n_red_tiles = (unsigned)((B + kReduceTile - 1) / kReduceTile);
     if (c->n_red_tiles == 0) c->n_red_tiles = 1;
-    const unsigned nt = c->n_sel_tiles, nr = c->n_red_tiles;
+    const unsigned nr = c->n_red_tiles;
 
     rc = SCAR_OK;
     auto A = [&](auto **p, size_t bytes) {
@@ -434,14 +450,14 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     A(&c->d_shard_mask, g.n_shards);
     A(&c->d_block_mask, B);
     A(&c->st, sizeof(SelState));
-    A(&c->ta.gt, nt * 4);
-    A(&c->ta.eq, nt * 4);
-    A(&c->ta.nf, nt * 4);
-    A(&c->ta.len_gt, nt * 8);
-    A(&c->ta.len_eq, nt * 8);
-    A(&c->ta.eq_base, nt * 4);
-    A(&c->ta.sel_base, nt * 4);
-    A(&c->ta.len_base, nt * 8);
+    if (rc == SCAR_OK)
+        rc = dt == SCAR_F32 ? plan_select<unsigned, float>(c) : plan_select<unsigned long long, unsigned long long>(c);
+    const unsigned ng = c->sel_grid;
+    A(&c->ca.gt, ng * 4);
+    A(&c->ca.eq, ng * 4);
+    A(&c->ca.nf, ng * 4);
+    A(&c->ca.len_gt, ng * 8);
+    A(&c->ca.len_eq, ng * 8);
     A(&c->rt_sum, nr * 8);
     A(&c->rt_l1, nr * 8);
     A(&c->rt_blocks, nr * 8);
@@ -695,7 +711,7 @@ const char *scar_strerror(int code) {
         case SCAR_ERR_ALLOC: return "allocation failed";
         case SCAR_ERR_CUDA: return "CUDA runtime error";
         case SCAR_ERR_STATE: return "call not valid in this state";
-        case SCAR_ERR_TIMEOUT: return "device-side wait timed out";
+        case SCAR_ERR_TIMEOUT: return "a bounded device-side wait gave up";
         case SCAR_ERR_CAPACITY: return "problem exceeds a fixed-size internal buffer";
         default: return "unknown error";
     }

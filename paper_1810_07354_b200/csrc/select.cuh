@@ -8,17 +8,27 @@
 // non-negative float32 score (NaN and +Inf both map to the +Inf pattern, so
 // such blocks rank first), or the uint64 l1 score itself.
 //
-//   k_radix_pass x P   most-significant digit first; each CTA first resolves the
-//                      previous digit from the previous pass's global histogram
-//                      (every CTA repeats the same small scan), then histograms
-//                      its tile of keys that match the prefix so far
-//   k_select_count     resolves the last digit -> threshold key tau and `need`
-//                      (how many keys equal to tau are taken); per-tile counts;
-//                      the CTA that finishes last turns them into per-tile bases
-//   k_select_emit      ordered compaction into sel[] / poff[]
+// The whole selection is ONE kernel, launched cooperatively (every CTA is
+// resident), so its phases are separated by grid-wide barriers instead of
+// kernel boundaries: the score array is small (4-8 bytes per block), and five
+// to eight dependent launches cost more than the work itself.  Each CTA owns a
+// contiguous range of 2048-key tiles.
 //
-// No kernel waits on another CTA: cross-CTA order comes from kernel boundaries
-// and from a ticket counter whose last taker does the epilogue.
+//   digit passes   most-significant digit first: shared-memory histogram of
+//                  the keys that match the prefix so far, flushed with integer
+//                  atomics; barrier; every CTA resolves the digit from the
+//                  global histogram (the same small scan in every CTA).
+//                  Digits that are zero in every uint64 key are skipped.
+//   counts         with the threshold key tau and `need` (how many keys equal
+//                  to tau are taken): per-CTA counts and summed lengths of the
+//                  keys above / equal to tau; barrier; every CTA scans those
+//                  into its own output bases
+//   boundary       only when the tau-keys run out inside one CTA's range: that
+//                  CTA sums the lengths of the ones it takes; barrier
+//   emit           ordered compaction into sel[] / poff[]
+//
+// The barrier is a counter in global memory with a bounded spin: a CTA that
+// gives up records an error and leaves, and the host reports SCAR_ERR_TIMEOUT.
 #pragma once
 #include "block_pass.cuh"
 
@@ -26,15 +36,17 @@ namespace scar {
 
 constexpr int kMaxPasses = 6;
 constexpr int kHistBins = 2048;
-constexpr int kSelTile = 2048;  // keys per CTA in every selection kernel
+constexpr int kSelTile = 2048;  // keys per tile
 constexpr int kPerThread = kSelTile / kThreads;
+constexpr unsigned kBarrierSpinLimit = 1u << 21;  // x >= 64 ns per try: gives up after >= 0.13 s
 
 struct SelState {
     unsigned long long key_or;  // OR of all uint64 keys seen since the last selection
-    unsigned long long prefix[kMaxPasses];
-    unsigned long long remaining[kMaxPasses];
-    unsigned ticket_count;
-    unsigned ticket_reduce;
+    unsigned long long partial_len;  // summed length of the tau-blocks taken in the boundary CTA
+    unsigned barrier;           // arrivals at the grid barrier during the running selection
+    unsigned departed;          // CTAs that have passed their last barrier
+    unsigned error;             // non-zero once a barrier wait gave up
+    unsigned ticket_reduce;     // ticket of the perturbation-norm reduction (block_pass.cuh)
     unsigned hist[kMaxPasses][kHistBins];
 };
 
@@ -42,17 +54,16 @@ struct SaveInfoDev {
     unsigned long long k;
     unsigned long long payload_elems;
     unsigned long long nonfinite_blocks;
+    unsigned long long error;  // copy of SelState::error at the end of the selection
 };
 
-struct TileArrays {
-    unsigned *gt;               // keys > tau per tile
-    unsigned *eq;               // keys == tau per tile
-    unsigned *nf;               // non-finite scores per tile
+// One entry per CTA of the selection kernel.
+struct CtaArrays {
+    unsigned *gt;               // keys > tau
+    unsigned *eq;               // keys == tau
+    unsigned *nf;               // non-finite scores
     unsigned long long *len_gt; // summed block lengths of the above
     unsigned long long *len_eq;
-    unsigned *eq_base;          // exclusive scans written by the last CTA
-    unsigned *sel_base;
-    unsigned long long *len_base;
 };
 
 template <typename K> struct KeyTraits;
@@ -101,6 +112,36 @@ template <typename W> __device__ __forceinline__ W cta_excl_scan(W v, W *sh /*kT
     return before + inc - v;
 }
 
+// Grid-wide barrier number `phase` (1, 2, ...) of a cooperative launch: every
+// CTA of the grid must call it the same number of times.  Returns false when
+// the wait was abandoned (it cannot happen while all CTAs are resident, which a
+// cooperative launch guarantees; the bound is there so that nothing can hang).
+__device__ __forceinline__ bool grid_barrier(SelState *st, unsigned phase) {
+    __shared__ bool ok;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(&st->barrier, 1u);
+        const unsigned target = phase * gridDim.x;
+        volatile unsigned *ctr = &st->barrier;
+        volatile unsigned *err = &st->error;
+        bool good = true;
+        unsigned tries = 0;
+        while (*ctr < target) {
+            if (*err != 0 || ++tries > kBarrierSpinLimit) {
+                atomicExch(&st->error, 1u);
+                good = false;
+                break;
+            }
+            __nanosleep(64);
+        }
+        __threadfence();
+        ok = good;
+    }
+    __syncthreads();
+    return ok;
+}
+
 // Resolves one digit: scanning bins from the highest down, finds the bin d with
 //   count(bins > d) < remaining <= count(bins >= d)
 // and returns it; remaining becomes the rank wanted inside bin d.
@@ -111,7 +152,7 @@ __device__ __forceinline__ unsigned resolve_digit(const unsigned *hist, int widt
     unsigned local[kHistBins / kThreads];
     unsigned long long sum = 0;
     for (int i = 0; i < per; ++i) {
-        local[i] = hist[nb - 1 - (threadIdx.x * per + i)];
+        local[i] = __ldcg(hist + (nb - 1 - (threadIdx.x * per + i)));
         sum += local[i];
     }
     unsigned long long cum = cta_excl_scan<unsigned long long>(sum, sh_scan, nullptr);
@@ -130,73 +171,13 @@ __device__ __forceinline__ unsigned resolve_digit(const unsigned *hist, int widt
     return d;
 }
 
-// State after resolving passes 0..p-1, identical in every CTA.  p == 0: empty
-// prefix, remaining = k.  CTA 0 records the newly resolved digit for the next kernel.
-template <typename K>
-__device__ __forceinline__ void resolve_prefix(SelState *st, int p, unsigned long long k, unsigned long long key_or,
-                                               unsigned long long &prefix, unsigned long long &remaining,
-                                               unsigned long long *sh_scan, unsigned long long *sh_out) {
-    using KT = KeyTraits<K>;
-    prefix = 0;
-    remaining = k;
-    if (p == 0) return;
-    if (p >= 2) {
-        prefix = st->prefix[p - 2];
-        remaining = st->remaining[p - 2];
-    }
-    const int q = p - 1;
-    const unsigned long long mask = (1ull << KT::width(q)) - 1;
-    unsigned d = 0;
-    if (!KT::kSkippable || ((key_or >> KT::shift(q)) & mask) != 0)
-        d = resolve_digit(st->hist[q], KT::width(q), remaining, sh_scan, sh_out);
-    prefix = (prefix << KT::width(q)) | d;
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        st->prefix[q] = prefix;
-        st->remaining[q] = remaining;
-    }
-}
-
+// Flags of the kPerThread consecutive blocks a thread owns in tile t.
 template <typename K, typename S>
-__global__ void __launch_bounds__(kThreads)
-k_radix_pass(const S *__restrict__ score, unsigned long long n_blocks, unsigned long long k, int p, SelState *st) {
-    using KT = KeyTraits<K>;
-    __shared__ unsigned sh_hist[kHistBins];
-    __shared__ unsigned long long sh_scan[kThreads / 32 + 1];
-    __shared__ unsigned long long sh_out[2];
-    const unsigned long long key_or = KT::kSkippable ? st->key_or : ~0ull;
-    unsigned long long prefix, remaining;
-    resolve_prefix<K>(st, p, k, key_or, prefix, remaining, sh_scan, sh_out);
-    if (blockIdx.x == 0 && p + 1 < KT::kPasses)
-        for (int i = threadIdx.x; i < kHistBins; i += kThreads) st->hist[p + 1][i] = 0;
-    const int shift = KT::shift(p), width = KT::width(p);
-    const unsigned long long mask = (1ull << width) - 1;
-    if (KT::kSkippable && ((key_or >> shift) & mask) == 0) return;  // this digit is 0 in every key
-    for (int i = threadIdx.x; i < kHistBins; i += kThreads) sh_hist[i] = 0;
-    __syncthreads();
-    const unsigned long long base = (unsigned long long)blockIdx.x * kSelTile;
-#pragma unroll
-    for (int j = 0; j < kPerThread; ++j) {
-        unsigned long long i = base + threadIdx.x + (unsigned long long)j * kThreads;
-        if (i < n_blocks) {
-            K key = KT::key(score[i]);
-            bool match = p == 0 || ((unsigned long long)key >> (shift + width)) == prefix;
-            if (match) atomicAdd(&sh_hist[(unsigned)(((unsigned long long)key >> shift) & mask)], 1u);
-        }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < (1 << width); i += kThreads) {
-        unsigned c = sh_hist[i];
-        if (c) atomicAdd(&st->hist[p][i], c);
-    }
-}
-
-// Flags of the kPerThread consecutive blocks a thread owns in its tile.
-template <typename K, typename S>
-__device__ __forceinline__ void tile_flags(const S *__restrict__ score, unsigned long long n_blocks, bool none, K tau,
-                                           unsigned &gt_bits, unsigned &eq_bits, unsigned &nf_bits) {
+__device__ __forceinline__ void tile_flags(const S *__restrict__ score, unsigned long long n_blocks, unsigned t, bool none,
+                                           K tau, unsigned &gt_bits, unsigned &eq_bits, unsigned &nf_bits) {
     using KT = KeyTraits<K>;
     gt_bits = eq_bits = nf_bits = 0;
-    const unsigned long long first = (unsigned long long)blockIdx.x * kSelTile + (unsigned long long)threadIdx.x * kPerThread;
+    const unsigned long long first = (unsigned long long)t * kSelTile + (unsigned long long)threadIdx.x * kPerThread;
 #pragma unroll
     for (int j = 0; j < kPerThread; ++j) {
         unsigned long long b = first + j;
@@ -213,173 +194,238 @@ __device__ __forceinline__ void tile_flags(const S *__restrict__ score, unsigned
 
 template <typename K, typename S>
 __global__ void __launch_bounds__(kThreads)
-k_select_count(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st, TileArrays ta,
-               SaveInfoDev *info, unsigned long long *poff) {
+k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st, CtaArrays ca, SaveInfoDev *info,
+         uint32_t *__restrict__ sel, unsigned long long *__restrict__ poff, unsigned n_tiles, unsigned tiles_per_cta) {
     using KT = KeyTraits<K>;
-    __shared__ unsigned long long sh_scan[kThreads / 32 + 1];
-    __shared__ unsigned long long sh_out[2];
-    __shared__ unsigned long long sh_red[kThreads / 32];
-    __shared__ bool is_last;
+    typedef unsigned long long u64;
+    __shared__ unsigned sh_hist[kHistBins];
+    __shared__ u64 sh_scan[kThreads / 32 + 1];
+    __shared__ u64 sh_out[2];
+    __shared__ u64 sh_red[kThreads / 32];
     __shared__ long long sh_boundary;
+    __shared__ u64 sh_boundary_take;
+    __shared__ bool sh_last;
+
+    const u64 B = g.n_blocks;
+    const unsigned t_lo = blockIdx.x * tiles_per_cta;
+    const unsigned t_hi = t_lo + tiles_per_cta < n_tiles ? t_lo + tiles_per_cta : n_tiles;
     const bool none = k == 0;
-    unsigned long long prefix = 0, need = 0;
+    const u64 key_or = KT::kSkippable ? st->key_or : ~0ull;  // reset only after the last barrier
+    unsigned phase = 0;
+    bool alive = true;
+
+    // ---- digit passes: tau = the k-th largest key, need = how many keys equal to tau are taken
+    u64 prefix = 0, need = k;
     if (!none) {
-        const unsigned long long key_or = KT::kSkippable ? st->key_or : ~0ull;
-        resolve_prefix<K>(st, KT::kPasses, k, key_or, prefix, need, sh_scan, sh_out);
+        for (int p = 0; p < KT::kPasses && alive; ++p) {
+            const int shift = KT::shift(p), width = KT::width(p);
+            const u64 mask = (1ull << width) - 1;
+            if (KT::kSkippable && ((key_or >> shift) & mask) == 0) {  // this digit is 0 in every key
+                prefix <<= width;
+                continue;
+            }
+            for (int i = threadIdx.x; i < kHistBins; i += kThreads) sh_hist[i] = 0;
+            __syncthreads();
+            for (unsigned t = t_lo; t < t_hi; ++t) {
+                const u64 base = (u64)t * kSelTile;
+#pragma unroll
+                for (int j = 0; j < kPerThread; ++j) {
+                    const u64 i = base + threadIdx.x + (u64)j * kThreads;
+                    if (i < B) {
+                        const K key = KT::key(score[i]);
+                        const bool match = p == 0 || ((u64)key >> (shift + width)) == prefix;
+                        if (match) atomicAdd(&sh_hist[(unsigned)(((u64)key >> shift) & mask)], 1u);
+                    }
+                }
+            }
+            __syncthreads();
+            for (int i = threadIdx.x; i < (1 << width); i += kThreads) {
+                const unsigned c = sh_hist[i];
+                if (c) atomicAdd(&st->hist[p][i], c);
+            }
+            alive = grid_barrier(st, ++phase);
+            if (alive) prefix = (prefix << width) | resolve_digit(st->hist[p], width, need, sh_scan, sh_out);
+        }
     }
     const K tau = (K)prefix;
-    unsigned gt_bits, eq_bits, nf_bits;
-    tile_flags<K, S>(score, g.n_blocks, none, tau, gt_bits, eq_bits, nf_bits);
-    unsigned long long lgt = 0, leq = 0;
-    const unsigned long long first = (unsigned long long)blockIdx.x * kSelTile + (unsigned long long)threadIdx.x * kPerThread;
-    for (int j = 0; j < kPerThread; ++j)
-        if ((gt_bits | eq_bits) >> j & 1u) {
-            uint64_t beg, len;
-            g.range((uint32_t)(first + j), beg, len);
-            if (gt_bits >> j & 1u) lgt += len; else leq += len;
-        }
-    unsigned long long c_gt = cta_sum<unsigned long long>(__popc(gt_bits), sh_red);
-    unsigned long long c_eq = cta_sum<unsigned long long>(__popc(eq_bits), sh_red);
-    unsigned long long c_nf = cta_sum<unsigned long long>(__popc(nf_bits), sh_red);
-    lgt = cta_sum<unsigned long long>(lgt, sh_red);
-    leq = cta_sum<unsigned long long>(leq, sh_red);
-    if (threadIdx.x == 0) {
-        ta.gt[blockIdx.x] = (unsigned)c_gt;
-        ta.eq[blockIdx.x] = (unsigned)c_eq;
-        ta.nf[blockIdx.x] = (unsigned)c_nf;
-        ta.len_gt[blockIdx.x] = lgt;
-        ta.len_eq[blockIdx.x] = leq;
-        __threadfence();
-        is_last = atomicAdd(&st->ticket_count, 1u) == gridDim.x - 1;
-        sh_boundary = -1;
-    }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
 
-    const unsigned nt = gridDim.x;
-    volatile unsigned *v_gt = ta.gt, *v_eq = ta.eq, *v_nf = ta.nf;
-    volatile unsigned long long *v_lgt = ta.len_gt, *v_leq = ta.len_eq;
-
-    // A: ranks of the tau-keys before each tile; find the tile where `need` runs out mid-tile.
-    unsigned long long carry = 0, nf_total = 0;
-    for (unsigned c = 0; c < nt; c += kThreads) {
-        unsigned t = c + threadIdx.x;
-        unsigned long long e = t < nt ? v_eq[t] : 0, tot;
-        unsigned long long ex = carry + cta_excl_scan<unsigned long long>(e, sh_scan, &tot);
-        if (t < nt) {
-            ta.eq_base[t] = (unsigned)ex;
-            if (ex < need && need < ex + e) sh_boundary = t;
-            nf_total += v_nf[t];
-        }
-        carry += tot;
-        __syncthreads();
-    }
-    nf_total = cta_sum<unsigned long long>(nf_total, sh_red);
-    __syncthreads();
-    const long long tb = sh_boundary;
-
-    // B: summed length of the tau-blocks actually taken inside the boundary tile.
-    unsigned long long partial_len = 0;
-    if (tb >= 0) {
-        const unsigned long long tfirst = (unsigned long long)tb * kSelTile + (unsigned long long)threadIdx.x * kPerThread;
-        unsigned eb = 0;
-        for (int j = 0; j < kPerThread; ++j) {
-            unsigned long long b = tfirst + j;
-            if (b < g.n_blocks && KT::key(score[b]) == tau) eb |= 1u << j;
-        }
-        unsigned long long rank = ta.eq_base[tb] + cta_excl_scan<unsigned long long>(__popc(eb), sh_scan, nullptr);
-        unsigned long long pl = 0;
-        for (int j = 0; j < kPerThread; ++j)
-            if (eb >> j & 1u) {
-                if (rank < need) {
+    // ---- counts over this CTA's tiles
+    u64 c_gt = 0, c_eq = 0, c_nf = 0, lgt = 0, leq = 0;
+    if (alive) {
+        for (unsigned t = t_lo; t < t_hi; ++t) {
+            unsigned gt_bits, eq_bits, nf_bits;
+            tile_flags<K, S>(score, B, t, none, tau, gt_bits, eq_bits, nf_bits);
+            const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kPerThread;
+            for (int j = 0; j < kPerThread; ++j)
+                if ((gt_bits | eq_bits) >> j & 1u) {
                     uint64_t beg, len;
-                    g.range((uint32_t)(tfirst + j), beg, len);
-                    pl += len;
+                    g.range((uint32_t)(first + j), beg, len);
+                    if (gt_bits >> j & 1u) lgt += len;
+                    else leq += len;
                 }
-                ++rank;
+            c_gt += __popc(gt_bits);
+            c_eq += __popc(eq_bits);
+            c_nf += __popc(nf_bits);
+        }
+        c_gt = cta_sum<u64>(c_gt, sh_red);
+        c_eq = cta_sum<u64>(c_eq, sh_red);
+        c_nf = cta_sum<u64>(c_nf, sh_red);
+        lgt = cta_sum<u64>(lgt, sh_red);
+        leq = cta_sum<u64>(leq, sh_red);
+        if (threadIdx.x == 0) {
+            ca.gt[blockIdx.x] = (unsigned)c_gt;
+            ca.eq[blockIdx.x] = (unsigned)c_eq;
+            ca.nf[blockIdx.x] = (unsigned)c_nf;
+            ca.len_gt[blockIdx.x] = lgt;
+            ca.len_eq[blockIdx.x] = leq;
+            sh_boundary = -1;
+            sh_boundary_take = 0;
+        }
+        alive = grid_barrier(st, ++phase);
+    }
+
+    // ---- every CTA scans the per-CTA counts into its own bases (the same scan in every CTA)
+    u64 my_eq_before = 0, my_sel_base = 0, my_len_base = 0, total_n = 0, total_l = 0, total_nf = 0;
+    long long cb = -1;
+    if (alive) {
+        u64 carry = 0, a_eq = 0, a_n = 0, a_l = 0, t_n = 0, t_l = 0, t_nf = 0;
+        for (unsigned c0 = 0; c0 < gridDim.x; c0 += kThreads) {
+            const unsigned c = c0 + threadIdx.x;
+            const bool in = c < gridDim.x;
+            const u64 e = in ? __ldcg(ca.eq + c) : 0;
+            u64 tot;
+            const u64 ex = carry + cta_excl_scan<u64>(e, sh_scan, &tot);
+            carry += tot;
+            if (in) {
+                u64 take = need > ex ? need - ex : 0;
+                if (take > e) take = e;
+                if (take != 0 && take != e) {  // the tau-keys run out inside this CTA's range
+                    sh_boundary = c;
+                    sh_boundary_take = take;
+                }
+                const u64 n = __ldcg(ca.gt + c) + take;
+                const u64 l = __ldcg(ca.len_gt + c) + (take == e ? __ldcg(ca.len_eq + c) : 0);
+                t_n += n;
+                t_l += l;
+                t_nf += __ldcg(ca.nf + c);
+                if (c < blockIdx.x) {
+                    a_eq += e;
+                    a_n += n;
+                    a_l += l;
+                }
             }
-        partial_len = cta_sum<unsigned long long>(pl, sh_red);
+        }
+        my_eq_before = cta_sum<u64>(a_eq, sh_red);
+        my_sel_base = cta_sum<u64>(a_n, sh_red);
+        my_len_base = cta_sum<u64>(a_l, sh_red);
+        total_n = cta_sum<u64>(t_n, sh_red);
+        total_l = cta_sum<u64>(t_l, sh_red);
+        total_nf = cta_sum<u64>(t_nf, sh_red);
         __syncthreads();
+        cb = sh_boundary;
     }
 
-    // C: per-tile output bases.
-    unsigned long long carry_n = 0, carry_l = 0;
-    for (unsigned c = 0; c < nt; c += kThreads) {
-        unsigned t = c + threadIdx.x;
-        unsigned long long n = 0, l = 0, tot_n, tot_l;
-        if (t < nt) {
-            unsigned long long e = v_eq[t], ex = ta.eq_base[t];
-            unsigned long long take = need > ex ? need - ex : 0;
-            if (take > e) take = e;
-            n = v_gt[t] + take;
-            l = v_lgt[t];
-            if (take == e) l += v_leq[t];
-            else if (take != 0) l += partial_len;
+    // ---- boundary CTA: summed length of the tau-blocks it takes (lowest ids first)
+    if (alive && cb >= 0) {  // the same decision in every CTA
+        if ((long long)blockIdx.x == cb) {
+            const u64 take = sh_boundary_take;
+            u64 run = 0, pl = 0;
+            for (unsigned t = t_lo; t < t_hi; ++t) {
+                unsigned gt_bits, eq_bits, nf_bits;
+                tile_flags<K, S>(score, B, t, false, tau, gt_bits, eq_bits, nf_bits);
+                u64 tot;
+                u64 rank = run + cta_excl_scan<u64>(__popc(eq_bits), sh_scan, &tot);
+                run += tot;
+                const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kPerThread;
+                for (int j = 0; j < kPerThread; ++j)
+                    if (eq_bits >> j & 1u) {
+                        if (rank < take) {
+                            uint64_t beg, len;
+                            g.range((uint32_t)(first + j), beg, len);
+                            pl += len;
+                        }
+                        ++rank;
+                    }
+            }
+            pl = cta_sum<u64>(pl, sh_red);
+            if (threadIdx.x == 0) st->partial_len = pl;
         }
-        unsigned long long exn = carry_n + cta_excl_scan<unsigned long long>(n, sh_scan, &tot_n);
-        unsigned long long exl = carry_l + cta_excl_scan<unsigned long long>(l, sh_scan, &tot_l);
-        if (t < nt) {
-            ta.sel_base[t] = (unsigned)exn;
-            ta.len_base[t] = exl;
+        alive = grid_barrier(st, ++phase);
+        if (alive) {
+            const u64 pl = __ldcg(&st->partial_len);
+            total_l += pl;
+            if ((long long)blockIdx.x > cb) my_len_base += pl;
         }
-        carry_n += tot_n;
-        carry_l += tot_l;
-        __syncthreads();
     }
+
+    // ---- emit: ordered compaction of this CTA's tiles
+    if (alive && !none) {
+        u64 run_eq = my_eq_before, pos_base = my_sel_base, off_base = my_len_base;
+        for (unsigned t = t_lo; t < t_hi; ++t) {
+            unsigned gt_bits, eq_bits, nf_bits;
+            tile_flags<K, S>(score, B, t, false, tau, gt_bits, eq_bits, nf_bits);
+            u64 tot_eq, tot_n, tot_l;
+            u64 rank = run_eq + cta_excl_scan<u64>(__popc(eq_bits), sh_scan, &tot_eq);
+            unsigned take_bits = gt_bits;
+            for (int j = 0; j < kPerThread; ++j)
+                if (eq_bits >> j & 1u) {
+                    if (rank < need) take_bits |= 1u << j;
+                    ++rank;
+                }
+            const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kPerThread;
+            u64 lens[kPerThread];
+            u64 lsum = 0;
+#pragma unroll
+            for (int j = 0; j < kPerThread; ++j) {
+                lens[j] = 0;
+                if (take_bits >> j & 1u) {
+                    uint64_t beg, len;
+                    g.range((uint32_t)(first + j), beg, len);
+                    lens[j] = len;
+                    lsum += len;
+                }
+            }
+            u64 pos = pos_base + cta_excl_scan<u64>(__popc(take_bits), sh_scan, &tot_n);
+            u64 off = off_base + cta_excl_scan<u64>(lsum, sh_scan, &tot_l);
+#pragma unroll
+            for (int j = 0; j < kPerThread; ++j)
+                if (take_bits >> j & 1u) {
+                    sel[pos] = (uint32_t)(first + j);
+                    poff[pos] = off;
+                    ++pos;
+                    off += lens[j];
+                }
+            run_eq += tot_eq;
+            pos_base += tot_n;
+            off_base += tot_l;
+        }
+    }
+    if (alive && blockIdx.x == 0 && threadIdx.x == 0) {
+        info->k = total_n;
+        info->payload_elems = total_l;
+        info->nonfinite_blocks = total_nf;
+        poff[total_n] = total_l;
+    }
+
+    // ---- the CTA that leaves last puts the shared state back for the next selection
+    __syncthreads();
     if (threadIdx.x == 0) {
-        info->k = carry_n;
-        info->payload_elems = carry_l;
-        info->nonfinite_blocks = nf_total;
-        poff[carry_n] = carry_l;
-        st->ticket_count = 0;
+        __threadfence();
+        sh_last = atomicAdd(&st->departed, 1u) == gridDim.x - 1;
     }
-}
-
-template <typename K, typename S>
-__global__ void __launch_bounds__(kThreads)
-k_select_emit(const S *__restrict__ score, Geom g, SelState *st, TileArrays ta, uint32_t *__restrict__ sel,
-              unsigned long long *__restrict__ poff) {
-    using KT = KeyTraits<K>;
-    __shared__ unsigned long long sh_scan[kThreads / 32 + 1];
-    const K tau = (K)st->prefix[KT::kPasses - 1];
-    const unsigned long long need = st->remaining[KT::kPasses - 1];
-    unsigned gt_bits, eq_bits, nf_bits;
-    tile_flags<K, S>(score, g.n_blocks, false, tau, gt_bits, eq_bits, nf_bits);
-    unsigned long long rank =
-        ta.eq_base[blockIdx.x] + cta_excl_scan<unsigned long long>(__popc(eq_bits), sh_scan, nullptr);
-    unsigned take_bits = gt_bits;
-    for (int j = 0; j < kPerThread; ++j)
-        if (eq_bits >> j & 1u) {
-            if (rank < need) take_bits |= 1u << j;
-            ++rank;
-        }
-    const unsigned long long first = (unsigned long long)blockIdx.x * kSelTile + (unsigned long long)threadIdx.x * kPerThread;
-    unsigned long long lens[kPerThread];
-    unsigned long long lsum = 0;
-#pragma unroll
-    for (int j = 0; j < kPerThread; ++j) {
-        lens[j] = 0;
-        if (take_bits >> j & 1u) {
-            uint64_t beg, len;
-            g.range((uint32_t)(first + j), beg, len);
-            lens[j] = len;
-            lsum += len;
-        }
+    __syncthreads();
+    if (!sh_last) return;
+    __threadfence();
+    for (int p = 0; p < KT::kPasses; ++p)
+        for (int i = threadIdx.x; i < kHistBins; i += kThreads) st->hist[p][i] = 0;
+    if (threadIdx.x == 0) {
+        const unsigned err = *reinterpret_cast<volatile unsigned *>(&st->error);
+        info->error = err;
+        st->key_or = 0;  // forget which uint64 key bits were seen
+        st->barrier = 0;
+        st->departed = 0;
+        st->error = 0;
     }
-    unsigned long long pos =
-        ta.sel_base[blockIdx.x] + cta_excl_scan<unsigned long long>(__popc(take_bits), sh_scan, nullptr);
-    unsigned long long off = ta.len_base[blockIdx.x] + cta_excl_scan<unsigned long long>(lsum, sh_scan, nullptr);
-#pragma unroll
-    for (int j = 0; j < kPerThread; ++j)
-        if (take_bits >> j & 1u) {
-            sel[pos] = (uint32_t)(first + j);
-            poff[pos] = off;
-            ++pos;
-            off += lens[j];
-        }
-    // Selection is over: forget which uint64 key bits were seen.
-    if (blockIdx.x == 0 && threadIdx.x == 0) st->key_or = 0;
 }
 
 }  // namespace scar

@@ -414,7 +414,7 @@ def test_launch_count_profile_and_last_info():
     api.scar_ckpt_profile(ck.ctx, True)
     assert ck.priority_save(0.25, sync=False) is None
     n1 = api.scar_ckpt_launch_count(ck.ctx)
-    assert n1 - n0 == 1 + 3 + 2 + 1  # scores, three radix passes, count + emit, pack
+    assert n1 - n0 == 1 + 1 + 1  # scores, the one selection kernel, pack
     ms = api.scar_ckpt_profile_read(ck.ctx)
     assert ms[0] > 0 and ms[1] > 0 and ms[2] > 0 and ms[3] == 0 and ms[4] == 0
     ck.recover_partial(w.lost_shards, sync=False)
