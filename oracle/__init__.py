@@ -206,6 +206,32 @@ def priority_save(x: np.ndarray, z: np.ndarray, boff: np.ndarray, r: Optional[fl
     return SaveResult(k, scores, sel, poff, payload, z_after, bad)
 
 
+# ---- baseline selectors of Section 5.4 ---------------------------------------------
+
+
+def select_round(n_blocks: int, k: int, cursor: int):
+    """`round`: the k blocks that follow the cursor, wrapping; returns (ascending ids, next cursor)."""
+    assert 0 <= k <= n_blocks and (0 <= cursor < n_blocks or (n_blocks == 0 and cursor == 0))
+    ids = [(cursor + j) % n_blocks for j in range(k)]
+    nxt = (cursor + k) % n_blocks if n_blocks else 0
+    return np.array(sorted(ids), dtype=np.uint32), nxt
+
+
+def select_random(priorities: np.ndarray, k: int) -> np.ndarray:
+    """`random`: the k blocks with the largest caller-drawn uint32 priorities, ties to the lowest id."""
+    _chk(priorities, np.uint32)
+    sel, _ = select_top_k(priorities.astype(np.uint64), k)
+    return sel
+
+
+def save_selected(x: np.ndarray, z: np.ndarray, boff: np.ndarray, sel: np.ndarray) -> SaveResult:
+    """Checkpoint step 4 of Section 4.3 for an id list chosen by any selector; scores are not computed."""
+    payload, poff = pack(x, boff, sel)
+    z_after = z.copy()
+    update(z_after, x, boff, sel)
+    return SaveResult(int(sel.size), np.empty(0), sel, poff, payload, z_after, 0)
+
+
 @dataclass
 class NormResult:
     l2: float  # sqrt of the fp64 sum of squares (float data); 0.0 for integer data

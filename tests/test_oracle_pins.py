@@ -491,6 +491,98 @@ def test_theorem_4_2_partition_identity_and_expectation():
     assert stderr < 0.05 * p * full, "the check has power"
 
 
+# ---- baseline selectors (Section 5.4) ---------------------------------------------------
+
+
+def test_round_robin_hand_cases():
+    sel, nxt = oracle.select_round(10, 4, 8)  # blocks 8, 9, 0, 1
+    assert sel.tolist() == [0, 1, 8, 9] and nxt == 2
+    sel, nxt = oracle.select_round(10, 4, 2)
+    assert sel.tolist() == [2, 3, 4, 5] and nxt == 6
+    sel, nxt = oracle.select_round(10, 10, 7)  # a full checkpoint leaves the cursor where it was
+    assert sel.tolist() == list(range(10)) and nxt == 7
+    sel, nxt = oracle.select_round(10, 0, 3)
+    assert sel.size == 0 and nxt == 3
+    sel, nxt = oracle.select_round(5, 5, 0)
+    assert sel.tolist() == [0, 1, 2, 3, 4] and nxt == 0
+
+
+@pytest.mark.parametrize("nb,k", [(97, 13), (64, 8), (10, 3), (7, 7), (1000, 1)])
+def test_round_robin_covers_every_block_once_per_cycle(nb, k):
+    # ceil(B/k) consecutive saves touch every block; before the wrap the selections are disjoint
+    cur, seen = 0, np.zeros(nb, dtype=np.int64)
+    for i in range(-(-nb // k)):
+        sel, cur = oracle.select_round(nb, k, cur)
+        assert sel.size == k and np.all(np.diff(sel.astype(np.int64)) > 0)
+        seen[sel] += 1
+    assert seen.min() >= 1 and seen.sum() == k * (-(-nb // k))
+    assert seen.max() <= 2 and (seen == 2).sum() == k * (-(-nb // k)) - nb
+    assert cur == (k * (-(-nb // k))) % nb
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_selector_matches_bruteforce_sort(seed):
+    r = rng(100 + seed)
+    nb = 500
+    pri = r.integers(0, 40 if seed % 2 else 2**32, size=nb, dtype=np.uint64).astype(np.uint32)  # odd seeds: many ties
+    for k in (0, 1, 17, 250, 499, 500):
+        want = sorted(sorted(range(nb), key=lambda b: (-int(pri[b]), b))[:k])
+        assert oracle.select_random(pri, k).tolist() == want
+    assert oracle.select_random(np.full(nb, 7, dtype=np.uint32), 9).tolist() == list(range(9))
+    assert oracle.select_random(np.array([0, 2**32 - 1, 5], dtype=np.uint32), 1).tolist() == [1]
+
+
+def test_random_selector_is_uniform_when_the_priorities_are():
+    # inclusion frequency of every block is k/B when the priorities are iid uniform
+    r = rng(7)
+    nb, k, trials = 40, 10, 4000
+    hits = np.zeros(nb)
+    for _ in range(trials):
+        hits[oracle.select_random(r.integers(0, 2**32, size=nb, dtype=np.uint64).astype(np.uint32), k)] += 1
+    p = k / nb
+    se = math.sqrt(p * (1 - p) / trials)
+    assert np.all(np.abs(hits / trials - p) < 4.5 * se)
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.int32])
+def test_baseline_saves_move_exactly_the_chosen_blocks(dtype):
+    x, z, boff = small_case(11, dtype)
+    nb = boff.size - 1
+    ids = block_ids(boff)
+    sel, _ = oracle.select_round(nb, 23, nb - 5)
+    res = oracle.save_selected(x, z, boff, sel)
+    chosen = np.isin(ids, sel)
+    assert res.payload.tobytes() == x[chosen].tobytes()
+    assert res.z_after[chosen].tobytes() == x[chosen].tobytes()
+    assert res.z_after[~chosen].tobytes() == z[~chosen].tobytes()
+    lens = (boff[1:] - boff[:-1])[sel.astype(np.int64)]
+    assert res.poff.tolist() == np.concatenate([[0], np.cumsum(lens)]).tolist()
+    # a round-robin cycle of full coverage ends in a full checkpoint
+    cur, zz = 0, z.copy()
+    for _ in range(-(-nb // 7)):
+        sel, cur = oracle.select_round(nb, 7, cur)
+        zz = oracle.save_selected(x, zz, boff, sel).z_after
+    assert zz.tobytes() == x.tobytes()
+
+
+def test_priority_beats_round_and_random_on_the_residual():
+    # Section 4.2's heuristic: for the same k the prioritized save leaves the smallest ||x - z||
+    x, z, boff = small_case(12, np.float32, nb=80)
+    nb = boff.size - 1
+    k = 20
+    full = oracle.perturbation_norm(x, z, boff).sumsq
+    pri = oracle.priority_save(x, z, boff, k=k)
+    best = oracle.perturbation_norm(x, pri.z_after, boff).sumsq
+    r = rng(13)
+    for trial in range(50):
+        sel, _ = oracle.select_round(nb, k, int(r.integers(0, nb)))
+        other = oracle.perturbation_norm(x, oracle.save_selected(x, z, boff, sel).z_after, boff).sumsq
+        assert best <= other * (1 + 1e-12) <= full * (1 + 1e-12)
+        sel = oracle.select_random(r.integers(0, 2**32, size=nb, dtype=np.uint64).astype(np.uint32), k)
+        other = oracle.perturbation_norm(x, oracle.save_selected(x, z, boff, sel).z_after, boff).sumsq
+        assert best <= other * (1 + 1e-12)
+
+
 def test_workload_recipes_have_the_stated_structure():
     w = make_workload("mlr", rows=16, cols=5000, seed=1)
     boff = block_offsets(w.geom)
