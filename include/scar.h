@@ -113,6 +113,27 @@ int scar_ckpt_priority_save(scar_ctx *ctx, double r, scar_save_info *out);
 /* Same with the block count given directly (0 <= k <= B). */
 int scar_ckpt_priority_save_k(scar_ctx *ctx, uint64_t k, scar_save_info *out);
 
+/* The two baseline selectors the paper compares the prioritized checkpoint with
+ * (Section 5.4).  Both skip the scoring pass (the score array keeps the values
+ * of the last scoring) and then pack the chosen blocks and refresh z on them
+ * exactly as a prioritized save does: same sel / poff / payload outputs, ids
+ * ascending.
+ *   round:  "selected in a round-robin manner": the k blocks that follow the
+ *           context's cursor, wrapping at the end of the buffer; the cursor
+ *           then advances by k (mod B).  It starts at block 0.
+ *   random: "selected uniformly at random".  The randomness is the caller's:
+ *           d_priorities is a DEVICE array of B uint32 values drawn
+ *           independently and uniformly by the caller; the k largest are taken,
+ *           ties to the lowest id, which is a uniform k-subset up to those ties.
+ *           Read when the enqueued work runs.
+ * 0 <= k <= B, otherwise SCAR_ERR_INVALID_ARG. */
+int scar_ckpt_save_round(scar_ctx *ctx, uint64_t k, scar_save_info *out);
+int scar_ckpt_save_random(scar_ctx *ctx, uint64_t k, const uint32_t *d_priorities, scar_save_info *out);
+
+/* Round-robin cursor: if set != NULL the cursor becomes *set (must be < B, or 0
+ * when B == 0); if get != NULL it receives the cursor.  Host state only. */
+int scar_ckpt_round_cursor(scar_ctx *ctx, const uint64_t *set, uint64_t *get);
+
 /* Partial recovery (Section 4.1; recovery step 2 of Section 4.3): for every
  * block of every lost shard, accumulates the perturbation of the appendix proof
  * of Theorem 4.1, ||z_S - x_S||, from the values x still holds, then overwrites

@@ -60,6 +60,9 @@ _SIGS = {
     "scar_ckpt_block_scores": (_int, [_vp]),
     "scar_ckpt_priority_save": (_int, [_vp, _dbl, C.POINTER(scar_save_info)]),
     "scar_ckpt_priority_save_k": (_int, [_vp, _u64, C.POINTER(scar_save_info)]),
+    "scar_ckpt_save_round": (_int, [_vp, _u64, C.POINTER(scar_save_info)]),
+    "scar_ckpt_save_random": (_int, [_vp, _u64, _vp, C.POINTER(scar_save_info)]),
+    "scar_ckpt_round_cursor": (_int, [_vp, C.POINTER(_u64), C.POINTER(_u64)]),
     "scar_recover_partial": (_int, [_vp, _vp, C.POINTER(scar_norm_info)]),
     "scar_recover_partial_blocks": (_int, [_vp, _vp, C.POINTER(scar_norm_info)]),
     "scar_perturbation_norm": (_int, [_vp, _vp, C.POINTER(scar_norm_info)]),
@@ -158,6 +161,28 @@ def scar_ckpt_priority_save_k(ctx: int, k: int, sync: bool = True) -> Optional[s
     _check(load_library().scar_ckpt_priority_save_k(ctx, k, C.byref(out) if sync else None),
            "scar_ckpt_priority_save_k")
     return out
+
+
+def scar_ckpt_save_round(ctx: int, k: int, sync: bool = True) -> Optional[scar_save_info]:
+    out = _save_out(sync)
+    _check(load_library().scar_ckpt_save_round(ctx, k, C.byref(out) if sync else None), "scar_ckpt_save_round")
+    return out
+
+
+def scar_ckpt_save_random(ctx: int, k: int, d_priorities, sync: bool = True) -> Optional[scar_save_info]:
+    out = _save_out(sync)
+    _check(load_library().scar_ckpt_save_random(ctx, k, _addr(d_priorities), C.byref(out) if sync else None),
+           "scar_ckpt_save_random")
+    return out
+
+
+def scar_ckpt_round_cursor(ctx: int, set_to: Optional[int] = None) -> int:
+    """Returns the round-robin cursor, after setting it when ``set_to`` is given."""
+    got = _u64(0)
+    new = _u64(set_to) if set_to is not None else None
+    _check(load_library().scar_ckpt_round_cursor(ctx, C.byref(new) if new is not None else None, C.byref(got)),
+           "scar_ckpt_round_cursor")
+    return int(got.value)
 
 
 def _norm_call(fn_name: str, ctx: int, mask, sync: bool) -> Optional[scar_norm_info]:
@@ -308,6 +333,15 @@ class ScarCheckpoint:
 
     def priority_save_k(self, k: int, sync: bool = True):
         return scar_ckpt_priority_save_k(self.ctx, k, sync)
+
+    def save_round(self, k: int, sync: bool = True):
+        return scar_ckpt_save_round(self.ctx, k, sync)
+
+    def save_random(self, k: int, d_priorities, sync: bool = True):
+        return scar_ckpt_save_random(self.ctx, k, d_priorities, sync)
+
+    def round_cursor(self, set_to: Optional[int] = None) -> int:
+        return scar_ckpt_round_cursor(self.ctx, set_to)
 
     def recover_partial(self, lost_shards: np.ndarray, sync: bool = True):
         return scar_recover_partial(self.ctx, lost_shards, sync)

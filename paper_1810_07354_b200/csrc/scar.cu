@@ -56,6 +56,7 @@ struct scar_ctx {
 
     std::vector<void *> owned;  // device allocations to free
     uint64_t launches = 0;
+    uint64_t round_cursor = 0;  // first block of the next round-robin save
 
     bool profile = false;
     cudaEvent_t ev[kNumEvents] = {};
@@ -183,12 +184,11 @@ template <typename T> void launch_scores(scar_ctx *c) {
 }
 
 // a2: one cooperative launch (all CTAs resident, so its grid-wide barriers cannot deadlock)
-template <typename K, typename S> int launch_select(scar_ctx *c, uint64_t k) {
-    const S *score = static_cast<const S *>(c->score);
+template <typename S> int launch_select(scar_ctx *c, const S *score, uint64_t k) {
     unsigned long long kk = k;
     unsigned nt = c->n_sel_tiles, per = c->sel_tiles_per_cta;
     void *args[] = {&score, &c->g, &kk, &c->st, &c->ca, &c->d_save, &c->sel, &c->poff, &nt, &per};
-    CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select<K, S>), dim3(c->sel_grid),
+    CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select<S>), dim3(c->sel_grid),
                                        dim3(kThreads), args, 0, c->stream));
     ++c->launches;
     return SCAR_OK;
@@ -196,11 +196,15 @@ template <typename K, typename S> int launch_select(scar_ctx *c, uint64_t k) {
 
 // Grid of the selection kernel: contiguous tile ranges over at most two CTAs per
 // SM (few enough that a barrier costs about a microsecond, and always resident).
-template <typename K, typename S> int plan_select(scar_ctx *c) {
-    int coop = 0, sms = 0, occ = 0;
+int plan_select(scar_ctx *c) {
+    int coop = 0, sms = 0, occ = 0, o = 0;
     CU_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
     CU_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device));
-    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_select<K, S>, kThreads, 0));
+    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_select<float>, kThreads, 0));
+    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, k_select<unsigned long long>, kThreads, 0));
+    occ = o < occ ? o : occ;
+    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, k_select<unsigned>, kThreads, 0));
+    occ = o < occ ? o : occ;
     if (!coop || sms < 1 || occ < 1) return SCAR_ERR_CUDA;
     const unsigned cap = (unsigned)sms * (unsigned)(occ < 2 ? occ : 2);
     const unsigned nt = c->n_sel_tiles;
@@ -309,9 +313,42 @@ int enqueue_save(scar_ctx *c, uint64_t k) {
     if (c->dt == SCAR_F32) launch_scores<float>(c);
     else launch_scores<int>(c);
     record(c, 1);
-    const int rc_sel = c->dt == SCAR_F32 ? launch_select<unsigned, float>(c, k)
-                                         : launch_select<unsigned long long, unsigned long long>(c, k);
+    const int rc_sel = c->dt == SCAR_F32
+                           ? launch_select<float>(c, static_cast<const float *>(c->score), k)
+                           : launch_select<unsigned long long>(c, static_cast<const unsigned long long *>(c->score), k);
     if (rc_sel != SCAR_OK) return rc_sel;
+    c->ran_select = true;
+    record(c, 2);
+    launch_pack(c, k);
+    c->ran_pack = k > 0;
+    record(c, 3);
+    CU_TRY(cudaGetLastError());
+    c->have_save = true;
+    return SCAR_OK;
+}
+
+// Saves with a selector that does not look at distances (Section 5.4: `round`, `random`):
+// no scoring pass; selection, then the same pack + cache refresh as a prioritized save.
+int enqueue_baseline_save(scar_ctx *c, uint64_t k, const uint32_t *d_priorities) {
+    c->last_call = 1;
+    c->ran_select = c->ran_pack = false;
+    record(c, 0);
+    record(c, 1);
+    if (c->g.n_blocks == 0) {
+        CU_TRY(cudaMemsetAsync(c->d_save, 0, sizeof(SaveInfoDev), c->stream));
+        CU_TRY(cudaMemsetAsync(c->poff, 0, sizeof(unsigned long long), c->stream));
+        c->have_save = true;
+        return SCAR_OK;
+    }
+    if (d_priorities) {
+        const int rc = launch_select<unsigned>(c, d_priorities, k);
+        if (rc != SCAR_OK) return rc;
+    } else {
+        const unsigned grid = (unsigned)((k + kThreads - 1) / kThreads);
+        k_select_round<<<grid ? grid : 1, kThreads, 0, c->stream>>>(c->g, c->round_cursor, k, c->sel, c->poff, c->d_save);
+        ++c->launches;
+        c->round_cursor = (c->round_cursor + k) % c->g.n_blocks;
+    }
     c->ran_select = true;
     record(c, 2);
     launch_pack(c, k);
@@ -451,7 +488,7 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     A(&c->d_block_mask, B);
     A(&c->st, sizeof(SelState));
     if (rc == SCAR_OK)
-        rc = dt == SCAR_F32 ? plan_select<unsigned, float>(c) : plan_select<unsigned long long, unsigned long long>(c);
+        rc = plan_select(c);
     const unsigned ng = c->sel_grid;
     A(&c->ca.gt, ng * 4);
     A(&c->ca.eq, ng * 4);
@@ -521,6 +558,34 @@ int scar_ckpt_priority_save(scar_ctx *c, double r, scar_save_info *out) {
     int rc = k_from_r(r, c->g.n_blocks, &k);
     if (rc != SCAR_OK) return rc;
     return scar_ckpt_priority_save_k(c, k, out);
+}
+
+int scar_ckpt_save_round(scar_ctx *c, uint64_t k, scar_save_info *out) {
+    if (!c || k > c->g.n_blocks) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    rc = enqueue_baseline_save(c, k, nullptr);
+    if (rc != SCAR_OK) return rc;
+    return out ? fetch_save(c, out) : SCAR_OK;
+}
+
+int scar_ckpt_save_random(scar_ctx *c, uint64_t k, const uint32_t *d_priorities, scar_save_info *out) {
+    if (!c || k > c->g.n_blocks || (!d_priorities && c->g.n_blocks)) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    rc = enqueue_baseline_save(c, k, d_priorities);
+    if (rc != SCAR_OK) return rc;
+    return out ? fetch_save(c, out) : SCAR_OK;
+}
+
+int scar_ckpt_round_cursor(scar_ctx *c, const uint64_t *set, uint64_t *get) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    if (set) {
+        if (c->g.n_blocks ? *set >= c->g.n_blocks : *set != 0) return SCAR_ERR_INVALID_ARG;
+        c->round_cursor = *set;
+    }
+    if (get) *get = c->round_cursor;
+    return SCAR_OK;
 }
 
 int scar_recover_partial(scar_ctx *c, const uint8_t *h_lost_shards, scar_norm_info *out) {

@@ -38,7 +38,7 @@ constexpr int kMaxPasses = 6;
 constexpr int kHistBins = 2048;
 constexpr int kSelTile = 2048;  // keys per tile
 constexpr int kPerThread = kSelTile / kThreads;
-constexpr unsigned kBarrierSpinLimit = 1u << 21;  // x >= 64 ns per try: gives up after >= 0.13 s
+constexpr unsigned kBarrierSpinLimit = 1u << 21;  // each try is a global load and a short sleep: gives up after >= 0.1 s
 
 struct SelState {
     unsigned long long key_or;  // OR of all uint64 keys seen since the last selection
@@ -66,17 +66,13 @@ struct CtaArrays {
     unsigned long long *len_eq;
 };
 
+// Digit plan per key width: 11/11/10 bits for 32-bit keys, 11/11/11/11/10/10 for 64-bit keys.
 template <typename K> struct KeyTraits;
 template <> struct KeyTraits<unsigned> {
     static constexpr int kPasses = 3;
     static constexpr bool kSkippable = false;
     __host__ __device__ static constexpr int shift(int p) { return p == 0 ? 21 : (p == 1 ? 10 : 0); }
     __host__ __device__ static constexpr int width(int p) { return p == 2 ? 10 : 11; }
-    static __device__ __forceinline__ unsigned key(float s) {
-        unsigned u = __float_as_uint(s) & 0x7fffffffu;
-        return u > 0x7f800000u ? 0x7f800000u : u;
-    }
-    static __device__ __forceinline__ bool nonfinite(unsigned k) { return k == 0x7f800000u; }
 };
 template <> struct KeyTraits<unsigned long long> {
     static constexpr int kPasses = 6;
@@ -85,8 +81,27 @@ template <> struct KeyTraits<unsigned long long> {
         return p == 0 ? 53 : p == 1 ? 42 : p == 2 ? 31 : p == 3 ? 20 : p == 4 ? 10 : 0;
     }
     __host__ __device__ static constexpr int width(int p) { return p >= 4 ? 10 : 11; }
-    static __device__ __forceinline__ unsigned long long key(unsigned long long s) { return s; }
-    static __device__ __forceinline__ bool nonfinite(unsigned long long) { return false; }
+};
+
+// What is ranked -> its order-preserving unsigned key.
+template <typename S> struct ScoreKey;
+template <> struct ScoreKey<float> {  // squared l2 scores
+    using K = unsigned;
+    static __device__ __forceinline__ K key(float s) {
+        unsigned u = __float_as_uint(s) & 0x7fffffffu;
+        return u > 0x7f800000u ? 0x7f800000u : u;
+    }
+    static __device__ __forceinline__ bool nonfinite(K k) { return k == 0x7f800000u; }
+};
+template <> struct ScoreKey<unsigned long long> {  // integer l1 scores
+    using K = unsigned long long;
+    static __device__ __forceinline__ K key(unsigned long long s) { return s; }
+    static __device__ __forceinline__ bool nonfinite(K) { return false; }
+};
+template <> struct ScoreKey<unsigned> {  // caller-supplied 32-bit priorities (random strategy)
+    using K = unsigned;
+    static __device__ __forceinline__ K key(unsigned s) { return s; }
+    static __device__ __forceinline__ bool nonfinite(K) { return false; }
 };
 
 // Exclusive prefix sum of one value per thread over the CTA; *total gets the sum.
@@ -121,19 +136,20 @@ __device__ __forceinline__ bool grid_barrier(SelState *st, unsigned phase) {
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
-        atomicAdd(&st->barrier, 1u);
         const unsigned target = phase * gridDim.x;
-        volatile unsigned *ctr = &st->barrier;
-        volatile unsigned *err = &st->error;
         bool good = true;
-        unsigned tries = 0;
-        while (*ctr < target) {
-            if (*err != 0 || ++tries > kBarrierSpinLimit) {
-                atomicExch(&st->error, 1u);
-                good = false;
-                break;
+        if (atomicAdd(&st->barrier, 1u) + 1 < target) {  // the last CTA to arrive does not wait
+            volatile unsigned *ctr = &st->barrier;
+            volatile unsigned *err = &st->error;
+            unsigned tries = 0;
+            while (*ctr < target) {
+                if (++tries > kBarrierSpinLimit || ((tries & 1023u) == 0 && *err != 0)) {
+                    atomicExch(&st->error, 1u);
+                    good = false;
+                    break;
+                }
+                __nanosleep(32);
             }
-            __nanosleep(64);
         }
         __threadfence();
         ok = good;
@@ -172,18 +188,20 @@ __device__ __forceinline__ unsigned resolve_digit(const unsigned *hist, int widt
 }
 
 // Flags of the kPerThread consecutive blocks a thread owns in tile t.
-template <typename K, typename S>
+template <typename S>
 __device__ __forceinline__ void tile_flags(const S *__restrict__ score, unsigned long long n_blocks, unsigned t, bool none,
-                                           K tau, unsigned &gt_bits, unsigned &eq_bits, unsigned &nf_bits) {
-    using KT = KeyTraits<K>;
+                                           typename ScoreKey<S>::K tau, unsigned &gt_bits, unsigned &eq_bits,
+                                           unsigned &nf_bits) {
+    using SK = ScoreKey<S>;
+    using K = typename SK::K;
     gt_bits = eq_bits = nf_bits = 0;
     const unsigned long long first = (unsigned long long)t * kSelTile + (unsigned long long)threadIdx.x * kPerThread;
 #pragma unroll
     for (int j = 0; j < kPerThread; ++j) {
         unsigned long long b = first + j;
         if (b < n_blocks) {
-            K key = KT::key(score[b]);
-            if (KT::nonfinite(key)) nf_bits |= 1u << j;
+            K key = SK::key(score[b]);
+            if (SK::nonfinite(key)) nf_bits |= 1u << j;
             if (!none) {
                 if (key > tau) gt_bits |= 1u << j;
                 else if (key == tau) eq_bits |= 1u << j;
@@ -192,10 +210,12 @@ __device__ __forceinline__ void tile_flags(const S *__restrict__ score, unsigned
     }
 }
 
-template <typename K, typename S>
+template <typename S>
 __global__ void __launch_bounds__(kThreads)
 k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st, CtaArrays ca, SaveInfoDev *info,
          uint32_t *__restrict__ sel, unsigned long long *__restrict__ poff, unsigned n_tiles, unsigned tiles_per_cta) {
+    using SK = ScoreKey<S>;
+    using K = typename SK::K;
     using KT = KeyTraits<K>;
     typedef unsigned long long u64;
     __shared__ unsigned sh_hist[kHistBins];
@@ -232,7 +252,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
                 for (int j = 0; j < kPerThread; ++j) {
                     const u64 i = base + threadIdx.x + (u64)j * kThreads;
                     if (i < B) {
-                        const K key = KT::key(score[i]);
+                        const K key = SK::key(score[i]);
                         const bool match = p == 0 || ((u64)key >> (shift + width)) == prefix;
                         if (match) atomicAdd(&sh_hist[(unsigned)(((u64)key >> shift) & mask)], 1u);
                     }
@@ -254,7 +274,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
     if (alive) {
         for (unsigned t = t_lo; t < t_hi; ++t) {
             unsigned gt_bits, eq_bits, nf_bits;
-            tile_flags<K, S>(score, B, t, none, tau, gt_bits, eq_bits, nf_bits);
+            tile_flags<S>(score, B, t, none, tau, gt_bits, eq_bits, nf_bits);
             const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kPerThread;
             for (int j = 0; j < kPerThread; ++j)
                 if ((gt_bits | eq_bits) >> j & 1u) {
@@ -332,7 +352,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
             u64 run = 0, pl = 0;
             for (unsigned t = t_lo; t < t_hi; ++t) {
                 unsigned gt_bits, eq_bits, nf_bits;
-                tile_flags<K, S>(score, B, t, false, tau, gt_bits, eq_bits, nf_bits);
+                tile_flags<S>(score, B, t, false, tau, gt_bits, eq_bits, nf_bits);
                 u64 tot;
                 u64 rank = run + cta_excl_scan<u64>(__popc(eq_bits), sh_scan, &tot);
                 run += tot;
@@ -363,7 +383,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
         u64 run_eq = my_eq_before, pos_base = my_sel_base, off_base = my_len_base;
         for (unsigned t = t_lo; t < t_hi; ++t) {
             unsigned gt_bits, eq_bits, nf_bits;
-            tile_flags<K, S>(score, B, t, false, tau, gt_bits, eq_bits, nf_bits);
+            tile_flags<S>(score, B, t, false, tau, gt_bits, eq_bits, nf_bits);
             u64 tot_eq, tot_n, tot_l;
             u64 rank = run_eq + cta_excl_scan<u64>(__popc(eq_bits), sh_scan, &tot_eq);
             unsigned take_bits = gt_bits;
@@ -425,6 +445,52 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
         st->barrier = 0;
         st->departed = 0;
         st->error = 0;
+    }
+}
+
+// ---- baseline strategies of Section 5.4 -------------------------------------
+//
+// `round`: the k blocks that follow a cursor, wrapping at the end of the buffer.
+// The id list stays ascending, so a wrapped selection is the run [0, wrap)
+// followed by the run [cursor, B); offsets inside a run of consecutive blocks
+// are differences of block start offsets, so no scan is needed.
+static __global__ void __launch_bounds__(kThreads)
+k_select_round(Geom g, unsigned long long cursor, unsigned long long k, uint32_t *__restrict__ sel,
+               unsigned long long *__restrict__ poff, SaveInfoDev *info) {
+    const unsigned long long j = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
+    if (k == 0) {
+        if (j == 0) {
+            poff[0] = 0;
+            info->k = 0;
+            info->payload_elems = 0;
+            info->nonfinite_blocks = 0;
+            info->error = 0;
+        }
+        return;
+    }
+    if (j >= k) return;
+    const unsigned long long B = g.n_blocks;
+    const unsigned long long wrap = cursor + k > B ? cursor + k - B : 0;  // ids below the cursor that are taken
+    uint64_t beg, len, first_beg, first_len, base = 0;
+    uint32_t b;
+    if (j < wrap) {
+        b = (uint32_t)j;
+        first_beg = 0;
+    } else {
+        b = (uint32_t)(cursor + (j - wrap));
+        g.range((uint32_t)cursor, first_beg, first_len);
+        if (wrap) g.range((uint32_t)wrap, base, first_len);  // elements of blocks [0, wrap)
+    }
+    g.range(b, beg, len);
+    const unsigned long long off = base + (beg - first_beg);
+    sel[j] = b;
+    poff[j] = off;
+    if (j == k - 1) {
+        poff[k] = off + len;
+        info->k = k;
+        info->payload_elems = off + len;
+        info->nonfinite_blocks = 0;
+        info->error = 0;
     }
 }
 
