@@ -223,6 +223,27 @@ uint64_t scar_ckpt_launch_count(const scar_ctx *ctx);
 int scar_ckpt_profile(scar_ctx *ctx, int enable);
 int scar_ckpt_profile_read(scar_ctx *ctx, float phase_ms[5]);
 
+/* ---- Iteration-cost arithmetic of Section 3 (host only, no GPU work) --------
+ * c is the linear convergence rate of the training algorithm, 0 < c < 1
+ * (Eq. 5/6); dist0 = ||x^(0) - x*|| > 0.  Every function returns NaN when an
+ * argument is outside its domain.
+ *
+ * baseline_iterations: kappa(x, eps) = log(dist0 / eps) / log(1 / c), the
+ *   iterations the unperturbed sequence needs to come within eps (Section 3.1).
+ * discounted_perturbation: Delta_T = sum_i c^(-iters[i]) * norms[i] of
+ *   Theorem 3.2, for n perturbations of size norms[i] >= 0 met at iteration
+ *   iters[i] (HOST arrays).  A single recovery at iteration T with
+ *   perturbation norm p gives c^(-T) * p.
+ * iteration_cost_bound: Theorem 3.2, log(1 + Delta_T / dist0) / log(1 / c):
+ *   the most extra iterations the perturbations can cost.
+ * irreducible_error: (c / (1 - c)) * delta_max, the accuracy floor when every
+ *   iteration may be perturbed by up to delta_max (Example 3.3, infinite
+ *   perturbations). */
+double scar_baseline_iterations(double dist0, double eps, double c);
+double scar_discounted_perturbation(const double *norms, const uint64_t *iters, uint64_t n, double c);
+double scar_iteration_cost_bound(double delta_T, double dist0, double c);
+double scar_irreducible_error(double delta_max, double c);
+
 /* Waits for the stream, frees everything the context owns (never x). */
 int scar_ckpt_destroy(scar_ctx *ctx);
 

@@ -270,3 +270,33 @@ def recover_partial(x, z, boff, lost_blocks):
     x_after = x.copy()
     res = _recover(x_after, z, boff, lost_blocks, write=True)
     return res, x_after
+
+
+# ---- iteration-cost arithmetic of Section 3 (plain Python floats, fp64) ---------------
+
+
+def baseline_iterations(dist0: float, eps: float, c: float) -> float:
+    """Section 3.1: iterations after which the unperturbed, linearly convergent sequence is eps-optimal."""
+    import math
+
+    return math.log(dist0 / eps) / math.log(1.0 / c)
+
+
+def discounted_perturbation(norms, iters, c: float) -> float:
+    """Theorem 3.2: ``Delta_T = sum_l c**(-l) * E||delta_l||`` over the perturbed iterations."""
+    total = 0.0
+    for nrm, l in zip(norms, iters):
+        total += float(nrm) / (c ** int(l))
+    return total
+
+
+def iteration_cost_bound(delta_T: float, dist0: float, c: float) -> float:
+    """Theorem 3.2: ``log(1 + Delta_T / ||x0 - x*||) / log(1 / c)``."""
+    import math
+
+    return math.log(1.0 + delta_T / dist0) / math.log(1.0 / c)
+
+
+def irreducible_error(delta_max: float, c: float) -> float:
+    """Example 3.3 (infinite perturbations): accuracy floor ``c / (1 - c) * Delta``."""
+    return c / (1.0 - c) * delta_max

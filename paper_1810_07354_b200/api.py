@@ -77,6 +77,10 @@ _SIGS = {
     "scar_ckpt_launch_count": (_u64, [_vp]),
     "scar_ckpt_profile": (_int, [_vp, _int]),
     "scar_ckpt_profile_read": (_int, [_vp, C.POINTER(C.c_float)]),
+    "scar_baseline_iterations": (_dbl, [_dbl, _dbl, _dbl]),
+    "scar_discounted_perturbation": (_dbl, [_vp, _vp, _u64, _dbl]),
+    "scar_iteration_cost_bound": (_dbl, [_dbl, _dbl, _dbl]),
+    "scar_irreducible_error": (_dbl, [_dbl, _dbl]),
     "scar_ckpt_destroy": (_int, [_vp]),
     "scar_strerror": (C.c_char_p, [_int]),
 }
@@ -267,6 +271,26 @@ def scar_ckpt_profile_read(ctx: int) -> list:
     ms = (C.c_float * 5)()
     _check(load_library().scar_ckpt_profile_read(ctx, ms), "scar_ckpt_profile_read")
     return list(ms)
+
+
+def scar_baseline_iterations(dist0: float, eps: float, c: float) -> float:
+    return float(load_library().scar_baseline_iterations(dist0, eps, c))
+
+
+def scar_discounted_perturbation(norms, iters, c: float) -> float:
+    nrm = np.ascontiguousarray(norms, dtype=np.float64)
+    its = np.ascontiguousarray(iters, dtype=np.uint64)
+    assert nrm.shape == its.shape and nrm.ndim == 1
+    return float(load_library().scar_discounted_perturbation(_addr(nrm) if nrm.size else None,
+                                                             _addr(its) if its.size else None, nrm.size, c))
+
+
+def scar_iteration_cost_bound(delta_T: float, dist0: float, c: float) -> float:
+    return float(load_library().scar_iteration_cost_bound(delta_T, dist0, c))
+
+
+def scar_irreducible_error(delta_max: float, c: float) -> float:
+    return float(load_library().scar_irreducible_error(delta_max, c))
 
 
 def scar_ckpt_destroy(ctx: int) -> None:
