@@ -193,6 +193,49 @@ int scar_ckpt_priority_save_host(scar_ctx *ctx, const void *h_x, double r, void 
                                  uint64_t *h_poff, scar_save_info *out);
 int scar_recover_partial_host(scar_ctx *ctx, void *h_x, const uint8_t *h_lost_shards, scar_norm_info *out);
 
+/* ---- Asynchronous drain of a save's output (Section 4.3) --------------------
+ * In the paper's protocol training resumes as soon as the in-memory cache (z)
+ * is refreshed, while the saved parameters go to persistent storage in the
+ * background, so the checkpoint overhead T_dump is only the prioritisation and
+ * the cache refresh.  Here: a save runs on the context's stream as always;
+ * scar_ckpt_drain_enqueue then copies that save's ids, offsets and payload to
+ * pinned host memory on a second, library-owned stream, ordered after the save
+ * by an event, and returns at once.  Two slots alternate, so the next save can
+ * run while the previous one is still being copied out.
+ *
+ *   drain_init     switches the context to drain mode and allocates the second
+ *                  device output set plus two pinned host mirrors.  From then
+ *                  on every save is limited to max_k blocks and to
+ *                  k * (longest block) <= max_payload_elems elements
+ *                  (SCAR_ERR_CAPACITY otherwise, nothing enqueued).  Waits for
+ *                  the context's stream.  Once per context.
+ *   drain_enqueue  hands the most recent save (there must be one that was not
+ *                  handed over yet: SCAR_ERR_STATE otherwise) to the drain
+ *                  stream; *ticket identifies it.  The next save writes to the
+ *                  other slot, and fails with SCAR_ERR_STATE, nothing enqueued,
+ *                  while that slot's ticket has not been released: at most two
+ *                  tickets are out at any time.  Does not wait.
+ *   drain_done     1 if the copy of that ticket has finished, 0 if not yet.
+ *   drain_wait     waits for the copy and fills *out with HOST pointers into
+ *                  the slot's pinned mirror: valid until drain_release.
+ *   drain_release  gives the slot back to the library (waits for the copy if it
+ *                  is still running).
+ * scar_ckpt_view keeps returning the device buffers of the most recent save.
+ * A save called with a non-NULL `out` fetches its result record over the same
+ * device-to-host path and can queue behind a running drain; to overlap, enqueue
+ * saves with out == NULL and read the record from the drained view. */
+typedef struct {
+    scar_save_info info;
+    const uint32_t *h_sel;  /* info.k ids, ascending */
+    const uint64_t *h_poff; /* info.k + 1 element offsets */
+    const void *h_payload;  /* info.payload_elems elements */
+} scar_drain_view;
+int scar_ckpt_drain_init(scar_ctx *ctx, uint64_t max_k, uint64_t max_payload_elems);
+int scar_ckpt_drain_enqueue(scar_ctx *ctx, uint64_t *ticket);
+int scar_ckpt_drain_done(scar_ctx *ctx, uint64_t ticket);
+int scar_ckpt_drain_wait(scar_ctx *ctx, uint64_t ticket, scar_drain_view *out);
+int scar_ckpt_drain_release(scar_ctx *ctx, uint64_t ticket);
+
 /* Replaces the running checkpoint by n_elems elements read from the device
  * buffer d_z_src (e.g. a checkpoint read back from storage).  Enqueue only. */
 int scar_ckpt_load(scar_ctx *ctx, const void *d_z_src);

@@ -43,6 +43,10 @@ class scar_norm_info(C.Structure):
     _fields_ = [("l2", C.c_double), ("l1", C.c_uint64), ("lost_blocks", C.c_uint64), ("lost_elems", C.c_uint64)]
 
 
+class scar_drain_view(C.Structure):
+    _fields_ = [("info", scar_save_info), ("h_sel", C.c_void_p), ("h_poff", C.c_void_p), ("h_payload", C.c_void_p)]
+
+
 def lib_path() -> str:
     return os.path.join(_PKG, "libscar.so")
 
@@ -70,6 +74,11 @@ _SIGS = {
     "scar_perturbation_norm_static": (_int, [_vp, _vp, _int, C.POINTER(scar_layout), _vp, _vp, _vp]),
     "scar_ckpt_priority_save_host": (_int, [_vp, _vp, _dbl, _vp, _vp, _vp, C.POINTER(scar_save_info)]),
     "scar_recover_partial_host": (_int, [_vp, _vp, _vp, C.POINTER(scar_norm_info)]),
+    "scar_ckpt_drain_init": (_int, [_vp, _u64, _u64]),
+    "scar_ckpt_drain_enqueue": (_int, [_vp, C.POINTER(_u64)]),
+    "scar_ckpt_drain_done": (_int, [_vp, _u64]),
+    "scar_ckpt_drain_wait": (_int, [_vp, _u64, C.POINTER(scar_drain_view)]),
+    "scar_ckpt_drain_release": (_int, [_vp, _u64]),
     "scar_ckpt_load": (_int, [_vp, _vp]),
     "scar_ckpt_last_info": (_int, [_vp, C.POINTER(scar_save_info), C.POINTER(scar_norm_info)]),
     "scar_ckpt_view": (_int, [_vp] + [C.POINTER(_vp)] * 5),
@@ -236,6 +245,44 @@ def scar_recover_partial_host(ctx: int, h_x, h_lost_shards: np.ndarray) -> scar_
     return out
 
 
+def scar_ckpt_drain_init(ctx: int, max_k: int, max_payload_elems: int) -> None:
+    _check(load_library().scar_ckpt_drain_init(ctx, max_k, max_payload_elems), "scar_ckpt_drain_init")
+
+
+def scar_ckpt_drain_enqueue(ctx: int) -> int:
+    t = _u64(0)
+    _check(load_library().scar_ckpt_drain_enqueue(ctx, C.byref(t)), "scar_ckpt_drain_enqueue")
+    return int(t.value)
+
+
+def scar_ckpt_drain_done(ctx: int, ticket: int) -> bool:
+    rc = load_library().scar_ckpt_drain_done(ctx, ticket)
+    if rc < 0:
+        raise ScarError(rc, "scar_ckpt_drain_done")
+    return bool(rc)
+
+
+def scar_ckpt_drain_wait(ctx: int, ticket: int, elem_dtype=np.float32) -> dict:
+    """Waits for the drain of ``ticket``; returns numpy views (no copy) of the pinned host mirror, valid until
+    ``scar_ckpt_drain_release``."""
+    v = scar_drain_view()
+    _check(load_library().scar_ckpt_drain_wait(ctx, ticket, C.byref(v)), "scar_ckpt_drain_wait")
+    k, n = int(v.info.k), int(v.info.payload_elems)
+
+    def view(addr, count, dt):
+        if count == 0:
+            return np.empty(0, dtype=dt)
+        buf = (C.c_char * (count * np.dtype(dt).itemsize)).from_address(addr)
+        return np.frombuffer(buf, dtype=dt, count=count)
+
+    return {"info": v.info, "sel": view(v.h_sel, k, np.uint32), "poff": view(v.h_poff, k + 1, np.uint64),
+            "payload": view(v.h_payload, n, elem_dtype)}
+
+
+def scar_ckpt_drain_release(ctx: int, ticket: int) -> None:
+    _check(load_library().scar_ckpt_drain_release(ctx, ticket), "scar_ckpt_drain_release")
+
+
 def scar_ckpt_load(ctx: int, d_z_src) -> None:
     _check(load_library().scar_ckpt_load(ctx, _addr(d_z_src)), "scar_ckpt_load")
 
@@ -378,6 +425,21 @@ class ScarCheckpoint:
 
     def perturbation_norm_blocks(self, d_lost_blocks=None, sync: bool = True):
         return scar_perturbation_norm_blocks(self.ctx, d_lost_blocks, sync)
+
+    def drain_init(self, max_k: int, max_payload_elems: int):
+        scar_ckpt_drain_init(self.ctx, max_k, max_payload_elems)
+
+    def drain_enqueue(self) -> int:
+        return scar_ckpt_drain_enqueue(self.ctx)
+
+    def drain_done(self, ticket: int) -> bool:
+        return scar_ckpt_drain_done(self.ctx, ticket)
+
+    def drain_wait(self, ticket: int) -> dict:
+        return scar_ckpt_drain_wait(self.ctx, ticket, np.float32 if self.dtype == SCAR_F32 else np.int32)
+
+    def drain_release(self, ticket: int):
+        scar_ckpt_drain_release(self.ctx, ticket)
 
     def load(self, d_z_src):
         scar_ckpt_load(self.ctx, d_z_src)

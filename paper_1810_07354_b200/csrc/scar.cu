@@ -24,6 +24,27 @@ constexpr int kNumEvents = 6;
 
 }  // namespace
 
+// Device buffers one save writes: payload, id list, offsets, result record.
+struct OutSet {
+    void *payload = nullptr;
+    uint32_t *sel = nullptr;
+    unsigned long long *poff = nullptr;
+    SaveInfoDev *info = nullptr;
+};
+
+// One of the two slots of the asynchronous drain (Section 4.3: the output to storage happens in the
+// background while training resumes): a device output set plus its pinned host mirror.
+struct DrainSlot {
+    OutSet dev{};
+    void *h_payload = nullptr;
+    uint32_t *h_sel = nullptr;
+    unsigned long long *h_poff = nullptr;
+    SaveInfoDev *h_info = nullptr;
+    cudaEvent_t saved = nullptr, drained = nullptr;
+    uint64_t k = 0, ticket = 0;
+    int state = 0;  // 0 free, 1 holds a save that was not handed to the drain, 2 draining, 3 host owns the buffers
+};
+
 struct scar_ctx {
     int device = 0;
     cudaStream_t stream = nullptr;
@@ -33,11 +54,10 @@ struct scar_ctx {
 
     void *x = nullptr;  // caller-owned
     void *z = nullptr;
-    void *payload = nullptr;
+    OutSet cur{};   // where the next save writes
+    OutSet last{};  // what the most recent save wrote (views and result fetches read this)
     void *score = nullptr;  // float[B] or uint64[B]
     void *part = nullptr;   // per-block perturbation partials, same type as score
-    uint32_t *sel = nullptr;
-    unsigned long long *poff = nullptr;
     uint64_t *d_boff = nullptr;
     uint8_t *d_shard_mask = nullptr;
     uint8_t *d_block_mask = nullptr;  // only used when a shard mask has too many runs
@@ -48,13 +68,21 @@ struct scar_ctx {
     double *rt_sum = nullptr;
     unsigned long long *rt_l1 = nullptr, *rt_blocks = nullptr, *rt_elems = nullptr;
     unsigned n_red_tiles = 0;
-    SaveInfoDev *d_save = nullptr;
     NormInfoDev *d_norm = nullptr;
     SaveInfoDev *h_save = nullptr;  // pinned
     NormInfoDev *h_norm = nullptr;  // pinned
     bool have_save = false, have_norm = false;
 
+    // asynchronous drain (off until scar_ckpt_drain_init)
+    bool drain = false;
+    DrainSlot slot[2];
+    int cur_slot = 0;
+    cudaStream_t drain_stream = nullptr;
+    uint64_t drain_cap_k = 0, drain_cap_elems = 0, next_ticket = 0;
+    uint64_t max_block_len = 0;
+
     std::vector<void *> owned;  // device allocations to free
+    std::vector<void *> owned_host;  // pinned host allocations to free
     uint64_t launches = 0;
     uint64_t round_cursor = 0;  // first block of the next round-robin save
 
@@ -187,7 +215,7 @@ template <typename T> void launch_scores(scar_ctx *c) {
 template <typename S> int launch_select(scar_ctx *c, const S *score, uint64_t k) {
     unsigned long long kk = k;
     unsigned nt = c->n_sel_tiles, per = c->sel_tiles_per_cta;
-    void *args[] = {&score, &c->g, &kk, &c->st, &c->ca, &c->d_save, &c->sel, &c->poff, &nt, &per};
+    void *args[] = {&score, &c->g, &kk, &c->st, &c->ca, &c->cur.info, &c->cur.sel, &c->cur.poff, &nt, &per};
     CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select<S>), dim3(c->sel_grid),
                                        dim3(kThreads), args, 0, c->stream));
     ++c->launches;
@@ -220,8 +248,8 @@ void launch_pack(scar_ctx *c, uint64_t k) {
         constexpr int G = decltype(gl)::value;
         constexpr bool VEC = decltype(vec)::value;
         k_pack_update<G, VEC><<<grid_for_groups(k, G), kThreads, 0, c->stream>>>(
-            static_cast<const uint32_t *>(c->x), static_cast<uint32_t *>(c->z), static_cast<uint32_t *>(c->payload),
-            c->g, c->sel, c->poff, k);
+            static_cast<const uint32_t *>(c->x), static_cast<uint32_t *>(c->z), static_cast<uint32_t *>(c->cur.payload),
+            c->g, c->cur.sel, c->cur.poff, k);
     });
     ++c->launches;
 }
@@ -266,12 +294,12 @@ int copy_elems(scar_ctx *c, void *dst, const void *src, uint64_t n) {
 }
 
 int fetch_save(scar_ctx *c, scar_save_info *out) {
-    CU_TRY(cudaMemcpyAsync(c->h_save, c->d_save, sizeof(SaveInfoDev), cudaMemcpyDeviceToHost, c->stream));
+    CU_TRY(cudaMemcpyAsync(c->h_save, c->last.info, sizeof(SaveInfoDev), cudaMemcpyDeviceToHost, c->stream));
     CU_TRY(cudaStreamSynchronize(c->stream));
     if (c->h_save->error) {
         // A grid barrier of the selection gave up; its outputs are not valid.  The kernel has
         // already put its barrier state back, so the context stays usable.
-        CU_TRY(cudaMemsetAsync(&c->d_save->error, 0, sizeof(unsigned long long), c->stream));
+        CU_TRY(cudaMemsetAsync(&c->last.info->error, 0, sizeof(unsigned long long), c->stream));
         return SCAR_ERR_TIMEOUT;
     }
     out->k = c->h_save->k;
@@ -300,13 +328,28 @@ int k_from_r(double r, uint64_t n_blocks, uint64_t *k) {
     return SCAR_OK;
 }
 
+// Common start of every save: in drain mode the save must fit the slot it writes to.
+int begin_save(scar_ctx *c, uint64_t k) {
+    if (c->drain) {
+        DrainSlot &sl = c->slot[c->cur_slot];
+        if (sl.state >= 2) return SCAR_ERR_STATE;  // both slots are still out: release the older ticket first
+        if (k > c->drain_cap_k || k * c->max_block_len > c->drain_cap_elems) return SCAR_ERR_CAPACITY;
+        sl.k = k;
+        sl.state = 1;
+    }
+    c->last = c->cur;
+    return SCAR_OK;
+}
+
 int enqueue_save(scar_ctx *c, uint64_t k) {
+    const int rc_begin = begin_save(c, k);
+    if (rc_begin != SCAR_OK) return rc_begin;
     c->last_call = 1;
     c->ran_select = c->ran_pack = false;
     record(c, 0);
     if (c->g.n_blocks == 0) {
-        CU_TRY(cudaMemsetAsync(c->d_save, 0, sizeof(SaveInfoDev), c->stream));
-        CU_TRY(cudaMemsetAsync(c->poff, 0, sizeof(unsigned long long), c->stream));
+        CU_TRY(cudaMemsetAsync(c->cur.info, 0, sizeof(SaveInfoDev), c->stream));
+        CU_TRY(cudaMemsetAsync(c->cur.poff, 0, sizeof(unsigned long long), c->stream));
         c->have_save = true;
         return SCAR_OK;
     }
@@ -330,13 +373,15 @@ int enqueue_save(scar_ctx *c, uint64_t k) {
 // Saves with a selector that does not look at distances (Section 5.4: `round`, `random`):
 // no scoring pass; selection, then the same pack + cache refresh as a prioritized save.
 int enqueue_baseline_save(scar_ctx *c, uint64_t k, const uint32_t *d_priorities) {
+    const int rc_begin = begin_save(c, k);
+    if (rc_begin != SCAR_OK) return rc_begin;
     c->last_call = 1;
     c->ran_select = c->ran_pack = false;
     record(c, 0);
     record(c, 1);
     if (c->g.n_blocks == 0) {
-        CU_TRY(cudaMemsetAsync(c->d_save, 0, sizeof(SaveInfoDev), c->stream));
-        CU_TRY(cudaMemsetAsync(c->poff, 0, sizeof(unsigned long long), c->stream));
+        CU_TRY(cudaMemsetAsync(c->cur.info, 0, sizeof(SaveInfoDev), c->stream));
+        CU_TRY(cudaMemsetAsync(c->cur.poff, 0, sizeof(unsigned long long), c->stream));
         c->have_save = true;
         return SCAR_OK;
     }
@@ -345,7 +390,8 @@ int enqueue_baseline_save(scar_ctx *c, uint64_t k, const uint32_t *d_priorities)
         if (rc != SCAR_OK) return rc;
     } else {
         const unsigned grid = (unsigned)((k + kThreads - 1) / kThreads);
-        k_select_round<<<grid ? grid : 1, kThreads, 0, c->stream>>>(c->g, c->round_cursor, k, c->sel, c->poff, c->d_save);
+        k_select_round<<<grid ? grid : 1, kThreads, 0, c->stream>>>(c->g, c->round_cursor, k, c->cur.sel, c->cur.poff,
+                                                                      c->cur.info);
         ++c->launches;
         c->round_cursor = (c->round_cursor + k) % c->g.n_blocks;
     }
@@ -430,7 +476,14 @@ int shard_set(scar_ctx *c, const uint8_t *h_lost_shards, LostSet &S) {
 
 void destroy_impl(scar_ctx *c) {
     cudaStreamSynchronize(c->stream);
+    if (c->drain_stream) cudaStreamSynchronize(c->drain_stream);
     for (void *p : c->owned) cudaFree(p);
+    for (void *p : c->owned_host) cudaFreeHost(p);
+    for (auto &sl : c->slot) {
+        if (sl.saved) cudaEventDestroy(sl.saved);
+        if (sl.drained) cudaEventDestroy(sl.drained);
+    }
+    if (c->drain_stream) cudaStreamDestroy(c->drain_stream);
     if (c->h_save) cudaFreeHost(c->h_save);
     if (c->h_norm) cudaFreeHost(c->h_norm);
     for (auto &e : c->ev)
@@ -465,6 +518,14 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     c->g = g;
     c->x = d_x;
     c->group_lanes = pick_group_lanes(g);
+    if (layout->block_offsets) {
+        for (uint64_t b = 0; b < g.n_blocks; ++b) {
+            const uint64_t len = layout->block_offsets[b + 1] - layout->block_offsets[b];
+            if (len > c->max_block_len) c->max_block_len = len;
+        }
+    } else {
+        c->max_block_len = g.row_len < g.block_elems ? g.row_len : g.block_elems;
+    }
 
     const uint64_t N = g.n_elems, B = g.n_blocks;
     const size_t score_bytes = (dt == SCAR_F32 ? 4 : 8) * B;
@@ -479,11 +540,11 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
         if (rc == SCAR_OK) rc = dev_alloc(c, p, bytes);
     };
     A(&c->z, N * 4);
-    A(&c->payload, N * 4);
+    A(&c->cur.payload, N * 4);
     A(&c->score, score_bytes);
     A(&c->part, score_bytes);
-    A(&c->sel, B * 4);
-    A(&c->poff, (B + 1) * 8);
+    A(&c->cur.sel, B * 4);
+    A(&c->cur.poff, (B + 1) * 8);
     A(&c->d_shard_mask, g.n_shards);
     A(&c->d_block_mask, B);
     A(&c->st, sizeof(SelState));
@@ -499,7 +560,7 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     A(&c->rt_l1, nr * 8);
     A(&c->rt_blocks, nr * 8);
     A(&c->rt_elems, nr * 8);
-    A(&c->d_save, sizeof(SaveInfoDev));
+    A(&c->cur.info, sizeof(SaveInfoDev));
     A(&c->d_norm, sizeof(NormInfoDev));
     if (rc == SCAR_OK && layout->block_offsets) A(&c->d_boff, (B + 1) * 8);
     if (rc == SCAR_OK && (cudaMallocHost(&c->h_save, sizeof(SaveInfoDev)) != cudaSuccess ||
@@ -507,10 +568,10 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
         rc = SCAR_ERR_ALLOC;
     if (rc == SCAR_OK) {
         bool ok = cudaMemsetAsync(c->st, 0, sizeof(SelState), c->stream) == cudaSuccess &&
-                  cudaMemsetAsync(c->d_save, 0, sizeof(SaveInfoDev), c->stream) == cudaSuccess &&
+                  cudaMemsetAsync(c->cur.info, 0, sizeof(SaveInfoDev), c->stream) == cudaSuccess &&
                   cudaMemsetAsync(c->d_norm, 0, sizeof(NormInfoDev), c->stream) == cudaSuccess &&
                   cudaMemsetAsync(c->score, 0, score_bytes ? score_bytes : 16, c->stream) == cudaSuccess &&
-                  cudaMemsetAsync(c->poff, 0, 8, c->stream) == cudaSuccess;
+                  cudaMemsetAsync(c->cur.poff, 0, 8, c->stream) == cudaSuccess;
         if (ok && layout->block_offsets) {
             ok = cudaMemcpyAsync(c->d_boff, layout->block_offsets, (B + 1) * 8, cudaMemcpyHostToDevice, c->stream) ==
                  cudaSuccess;
@@ -526,6 +587,7 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
         destroy_impl(c);
         return rc;
     }
+    c->last = c->cur;
     *out = c;
     return SCAR_OK;
 }
@@ -645,12 +707,12 @@ int scar_ckpt_priority_save_host(scar_ctx *c, const void *h_x, double r, void *h
     rc = enqueue_save(c, k);
     if (rc != SCAR_OK) return rc;
     // The id and offset lists have a size known up front; the payload length is data dependent.
-    if (k) CU_TRY(cudaMemcpyAsync(h_sel, c->sel, k * 4, cudaMemcpyDeviceToHost, c->stream));
-    CU_TRY(cudaMemcpyAsync(h_poff, c->poff, (k + 1) * 8, cudaMemcpyDeviceToHost, c->stream));
+    if (k) CU_TRY(cudaMemcpyAsync(h_sel, c->last.sel, k * 4, cudaMemcpyDeviceToHost, c->stream));
+    CU_TRY(cudaMemcpyAsync(h_poff, c->last.poff, (k + 1) * 8, cudaMemcpyDeviceToHost, c->stream));
     rc = fetch_save(c, out);
     if (rc != SCAR_OK) return rc;
     if (out->payload_elems) {
-        CU_TRY(cudaMemcpyAsync(h_payload, c->payload, out->payload_elems * 4, cudaMemcpyDeviceToHost, c->stream));
+        CU_TRY(cudaMemcpyAsync(h_payload, c->last.payload, out->payload_elems * 4, cudaMemcpyDeviceToHost, c->stream));
         CU_TRY(cudaStreamSynchronize(c->stream));
     }
     return SCAR_OK;
@@ -696,6 +758,127 @@ int scar_recover_partial_host(scar_ctx *c, void *h_x, const uint8_t *h_lost_shar
     return fetch_norm(c, out);
 }
 
+int scar_ckpt_drain_init(scar_ctx *c, uint64_t max_k, uint64_t max_payload_elems) {
+    if (!c || c->drain) return c ? SCAR_ERR_STATE : SCAR_ERR_INVALID_ARG;
+    if (max_k > c->g.n_blocks || max_payload_elems > c->g.n_elems) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    CU_TRY(cudaStreamSynchronize(c->stream));
+    const size_t pay = max_payload_elems * 4, ids = max_k * 4, offs = (max_k + 1) * 8;
+    DrainSlot &s0 = c->slot[0], &s1 = c->slot[1];
+    s0.dev = c->cur;  // slot 0 reuses the context's own output set
+    auto D = [&](auto **p, size_t bytes) {
+        if (rc == SCAR_OK) rc = dev_alloc(c, p, bytes);
+    };
+    auto H = [&](auto **p, size_t bytes) {
+        if (rc != SCAR_OK) return;
+        void *q = nullptr;
+        if (cudaMallocHost(&q, bytes ? bytes : 16) != cudaSuccess) {
+            cudaGetLastError();
+            rc = SCAR_ERR_ALLOC;
+            return;
+        }
+        c->owned_host.push_back(q);
+        *p = static_cast<std::remove_pointer_t<std::remove_reference_t<decltype(*p)>> *>(q);
+    };
+    D(&s1.dev.payload, pay);
+    D(&s1.dev.sel, ids);
+    D(&s1.dev.poff, offs);
+    D(&s1.dev.info, sizeof(SaveInfoDev));
+    for (auto &sl : c->slot) {
+        H(&sl.h_payload, pay);
+        H(&sl.h_sel, ids);
+        H(&sl.h_poff, offs);
+        H(&sl.h_info, sizeof(SaveInfoDev));
+        if (rc == SCAR_OK && (cudaEventCreateWithFlags(&sl.saved, cudaEventDisableTiming) != cudaSuccess ||
+                              cudaEventCreateWithFlags(&sl.drained, cudaEventDisableTiming) != cudaSuccess))
+            rc = SCAR_ERR_CUDA;
+    }
+    if (rc == SCAR_OK && cudaStreamCreateWithFlags(&c->drain_stream, cudaStreamNonBlocking) != cudaSuccess)
+        rc = SCAR_ERR_CUDA;
+    if (rc == SCAR_OK && (cudaMemsetAsync(s1.dev.info, 0, sizeof(SaveInfoDev), c->stream) != cudaSuccess ||
+                          cudaMemsetAsync(s1.dev.poff, 0, 8, c->stream) != cudaSuccess))
+        rc = SCAR_ERR_CUDA;
+    if (rc != SCAR_OK) {
+        cudaGetLastError();
+        return rc;  // what was allocated stays owned by the context and is freed by destroy
+    }
+    c->drain_cap_k = max_k;
+    c->drain_cap_elems = max_payload_elems;
+    c->cur_slot = 0;
+    c->drain = true;
+    return SCAR_OK;
+}
+
+int scar_ckpt_drain_enqueue(scar_ctx *c, uint64_t *ticket) {
+    if (!c || !ticket) return SCAR_ERR_INVALID_ARG;
+    if (!c->drain) return SCAR_ERR_STATE;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    DrainSlot &sl = c->slot[c->cur_slot];
+    if (sl.state != 1) return SCAR_ERR_STATE;
+    CU_TRY(cudaEventRecord(sl.saved, c->stream));
+    CU_TRY(cudaStreamWaitEvent(c->drain_stream, sl.saved, 0));
+    // The payload length is only known on the device; k * (longest block) bounds it and is known here.
+    uint64_t elems = sl.k * c->max_block_len;
+    if (elems > c->drain_cap_elems) elems = c->drain_cap_elems;
+    CU_TRY(cudaMemcpyAsync(sl.h_info, sl.dev.info, sizeof(SaveInfoDev), cudaMemcpyDeviceToHost, c->drain_stream));
+    if (sl.k) CU_TRY(cudaMemcpyAsync(sl.h_sel, sl.dev.sel, sl.k * 4, cudaMemcpyDeviceToHost, c->drain_stream));
+    CU_TRY(cudaMemcpyAsync(sl.h_poff, sl.dev.poff, (sl.k + 1) * 8, cudaMemcpyDeviceToHost, c->drain_stream));
+    if (elems) CU_TRY(cudaMemcpyAsync(sl.h_payload, sl.dev.payload, elems * 4, cudaMemcpyDeviceToHost, c->drain_stream));
+    CU_TRY(cudaEventRecord(sl.drained, c->drain_stream));
+    sl.state = 2;
+    sl.ticket = ++c->next_ticket;
+    *ticket = sl.ticket;
+    c->cur_slot = 1 - c->cur_slot;
+    c->cur = c->slot[c->cur_slot].dev;
+    return SCAR_OK;
+}
+
+static DrainSlot *slot_of(scar_ctx *c, uint64_t ticket) {
+    for (auto &sl : c->slot)
+        if (sl.state >= 2 && sl.ticket == ticket) return &sl;
+    return nullptr;
+}
+
+int scar_ckpt_drain_done(scar_ctx *c, uint64_t ticket) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    DrainSlot *sl = c->drain ? slot_of(c, ticket) : nullptr;
+    if (!sl) return SCAR_ERR_STATE;
+    if (sl->state == 3) return 1;
+    cudaError_t e = cudaEventQuery(sl->drained);
+    if (e == cudaSuccess) return 1;
+    if (e == cudaErrorNotReady) return 0;
+    cudaGetLastError();
+    return SCAR_ERR_CUDA;
+}
+
+int scar_ckpt_drain_wait(scar_ctx *c, uint64_t ticket, scar_drain_view *out) {
+    if (!c || !out) return SCAR_ERR_INVALID_ARG;
+    DrainSlot *sl = c->drain ? slot_of(c, ticket) : nullptr;
+    if (!sl) return SCAR_ERR_STATE;
+    CU_TRY(cudaEventSynchronize(sl->drained));
+    sl->state = 3;
+    if (sl->h_info->error) return SCAR_ERR_TIMEOUT;
+    out->info.k = sl->h_info->k;
+    out->info.payload_elems = sl->h_info->payload_elems;
+    out->info.nonfinite_blocks = sl->h_info->nonfinite_blocks;
+    out->h_sel = sl->h_sel;
+    out->h_poff = reinterpret_cast<const uint64_t *>(sl->h_poff);
+    out->h_payload = sl->h_payload;
+    return SCAR_OK;
+}
+
+int scar_ckpt_drain_release(scar_ctx *c, uint64_t ticket) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    DrainSlot *sl = c->drain ? slot_of(c, ticket) : nullptr;
+    if (!sl) return SCAR_ERR_STATE;
+    if (sl->state == 2) CU_TRY(cudaEventSynchronize(sl->drained));
+    sl->state = 0;
+    sl->ticket = 0;
+    return SCAR_OK;
+}
+
 int scar_ckpt_load(scar_ctx *c, const void *d_z_src) {
     if (!c || (!d_z_src && c->g.n_elems)) return SCAR_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(d_z_src) & 15) return SCAR_ERR_INVALID_ARG;
@@ -720,9 +903,9 @@ int scar_ckpt_view(scar_ctx *c, const void **d_z, const void **d_scores, const u
     if (!c) return SCAR_ERR_INVALID_ARG;
     if (d_z) *d_z = c->z;
     if (d_scores) *d_scores = c->score;
-    if (d_sel) *d_sel = c->sel;
-    if (d_poff) *d_poff = reinterpret_cast<const uint64_t *>(c->poff);
-    if (d_payload) *d_payload = c->payload;
+    if (d_sel) *d_sel = c->last.sel;
+    if (d_poff) *d_poff = reinterpret_cast<const uint64_t *>(c->last.poff);
+    if (d_payload) *d_payload = c->last.payload;
     return SCAR_OK;
 }
 
