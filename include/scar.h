@@ -43,6 +43,14 @@ typedef struct scar_ctx scar_ctx; /* opaque; created by scar_ckpt_init, freed by
  * (twice the length-scaled total variation that Appendix C uses for LDA). */
 typedef enum { SCAR_F32 = 0, SCAR_I32 = 1 } scar_dtype;
 
+/* Which norm measures the distance of a block to its saved copy.  DEFAULT is the
+ * one above for the element type.  L1 on SCAR_F32 data scores a block by
+ * sum |x_i - z_i| in float32 and reports perturbations as the plain sum (no
+ * square root): with per-block weights L_b / 2 this is the total variation of
+ * each topic distribution scaled by its document's length, the norm Appendix C
+ * uses for LDA.  On SCAR_I32 data L1 is the default already. */
+typedef enum { SCAR_NORM_DEFAULT = 0, SCAR_NORM_L1 = 1 } scar_norm;
+
 enum {
     SCAR_OK = 0,
     SCAR_ERR_INVALID_ARG = -1, /* NULL where not allowed, r outside [0,1], k > B, misaligned x ... */
@@ -81,7 +89,8 @@ typedef struct {
 } scar_save_info;
 
 typedef struct {
-    double l2;            /* SCAR_F32: ||z_S - x_S||_2 ; 0 for SCAR_I32 */
+    double l2;            /* SCAR_F32: ||z_S - x_S|| in the context's norm (l2 unless scar_ckpt_set_norm
+                             chose another); 0 for SCAR_I32 */
     uint64_t l1;          /* SCAR_I32: sum_{i in S} |z_i - x_i| ; 0 for SCAR_F32 */
     uint64_t lost_blocks; /* |S| in blocks */
     uint64_t lost_elems;  /* |S| in elements */
@@ -95,6 +104,18 @@ typedef struct {
  * current CUDA device.  cuda_stream is a cudaStream_t (NULL = default stream).
  * Waits for the stream before returning.  On error *out is NULL. */
 int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *layout, void *cuda_stream);
+
+/* Chooses the norm and optional per-block weights for all later scoring,
+ * selection and perturbation results of this context.  h_block_weights: HOST
+ * array of B finite floats >= 0 (copied before the call returns), or NULL for
+ * no weights; SCAR_F32 only (SCAR_ERR_INVALID_ARG with SCAR_I32: integer scores
+ * stay exact integers, and for count rows of fixed total the length-scaled
+ * total variation is half the plain l1 anyway).  With weights w a block scores
+ * w_b * dist(x_b, z_b) (dist = squared l2, or l1), and a perturbation is
+ * sqrt(sum_b w_b ||d_b||^2) or sum_b w_b ||d_b||_1, reported in the l2 field of
+ * scar_norm_info: a positive combination of block norms, hence a norm
+ * (Appendix C).  Waits for the stream. */
+int scar_ckpt_set_norm(scar_ctx *ctx, scar_norm norm, const float *h_block_weights);
 
 /* Checkpoint step 1 of Section 4.3 alone: recomputes score_b = dist(x_b, z_b)
  * for every block into the context's score array (float32 squared l2, or

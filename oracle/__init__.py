@@ -53,6 +53,7 @@ def _load():
                 "scar_oracle_layout_offsets": (None, [_u64, _u64, _u64, _p]),
                 "scar_oracle_expand_shards": (None, [_u64, _u64, _p, _p]),
                 "scar_oracle_scores_f32": (None, [_p, _p, _p, _u64, _p]),
+                "scar_oracle_scores_f32_l1": (None, [_p, _p, _p, _u64, _p]),
                 "scar_oracle_scores_i32": (None, [_p, _p, _p, _u64, _p]),
                 "scar_oracle_k_from_r": (_i64, [_dbl, _u64]),
                 "scar_oracle_select_f64": (_int, [_p, _u64, _u64, _p, _p]),
@@ -204,6 +205,48 @@ def priority_save(x: np.ndarray, z: np.ndarray, boff: np.ndarray, r: Optional[fl
     z_after = z.copy()
     update(z_after, x, boff, sel)
     return SaveResult(k, scores, sel, poff, payload, z_after, bad)
+
+
+# ---- other norms (Appendix C) -----------------------------------------------------
+
+
+def block_scores_norm(x: np.ndarray, z: np.ndarray, boff: np.ndarray, norm: str = "l2",
+                      weights: Optional[np.ndarray] = None) -> np.ndarray:
+    """fp64 block scores of float32 data under a weighted block norm: ``w_b * sum (x - z)^2`` (``"l2"``) or
+    ``w_b * sum |x - z|`` (``"l1"``; with ``w_b = L_b / 2`` the length-scaled total variation of Appendix C)."""
+    lib = _load()
+    _chk(x, np.float32), _chk(z, np.float32), _chk(boff, np.uint64)
+    nb = boff.size - 1
+    out = np.empty(nb, dtype=np.float64)
+    fn = {"l2": lib.scar_oracle_scores_f32, "l1": lib.scar_oracle_scores_f32_l1}[norm]
+    fn(_ptr(x), _ptr(z), _ptr(boff), nb, _ptr(out))
+    if weights is not None:
+        out = out * np.asarray(weights, dtype=np.float64)
+    return out
+
+
+def save_norm(x, z, boff, k: int, norm: str = "l2", weights=None) -> SaveResult:
+    """A prioritized save whose distances use the weighted norm above."""
+    scores = block_scores_norm(x, z, boff, norm, weights)
+    sel, bad = select_top_k(scores, k)
+    payload, poff = pack(x, boff, sel)
+    z_after = z.copy()
+    update(z_after, x, boff, sel)
+    return SaveResult(k, scores, sel, poff, payload, z_after, bad)
+
+
+def perturbation_norm_weighted(x, z, boff, lost_blocks=None, norm: str = "l2", weights=None) -> NormResult:
+    """Perturbation of recovering the lost blocks, in the weighted norm: the lost blocks' distances added up
+    (the supports are disjoint, proof of Theorem 4.1), square-rooted for l2.  Reported in the ``l2`` field."""
+    scores = block_scores_norm(x, z, boff, norm, weights)
+    nb = boff.size - 1
+    lost = np.ones(nb, dtype=bool) if lost_blocks is None else np.asarray(lost_blocks).astype(bool)
+    total = 0.0
+    for b in np.flatnonzero(lost):
+        total += float(scores[b])
+    lens = (boff[1:] - boff[:-1]).astype(np.int64)
+    value = float(np.sqrt(total)) if norm == "l2" else total
+    return NormResult(value, 0, total, int(lost.sum()), int(lens[lost].sum()))
 
 
 # ---- baseline selectors of Section 5.4 ---------------------------------------------

@@ -83,6 +83,20 @@ void scar_oracle_scores_f32(const float *x, const float *z, const uint64_t *boff
     }
 }
 
+/* Appendix C: for parameters that are distributions the distance is the total
+ * variation, (1/2) sum |x_i - z_i|, scaled per block; this is the plain l1 sum of
+ * float data, the scale (weight) is applied by the caller. */
+void scar_oracle_scores_f32_l1(const float *x, const float *z, const uint64_t *boff, uint64_t n_blocks,
+                               double *score)
+{
+    for (uint64_t b = 0; b < n_blocks; ++b) {
+        double acc = 0.0;
+        for (uint64_t i = boff[b]; i < boff[b + 1]; ++i)
+            acc += fabs((double)x[i] - (double)z[i]);
+        score[b] = acc;
+    }
+}
+
 /* Appendix C (LDA): distances between count rows use a length-scaled total
  * variation, which for counts is half the l1 distance; the factor 1/2 is
  * dropped so that score_b = sum_{i in b} |x_i - z_i| stays an integer. */

@@ -17,6 +17,7 @@ from typing import Optional
 import numpy as np
 
 SCAR_F32, SCAR_I32 = 0, 1
+SCAR_NORM_DEFAULT, SCAR_NORM_L1 = 0, 1
 SCAR_OK = 0
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
@@ -61,6 +62,7 @@ def exported_symbols() -> list:
 _vp, _u64, _int, _dbl = C.c_void_p, C.c_uint64, C.c_int, C.c_double
 _SIGS = {
     "scar_ckpt_init": (_int, [C.POINTER(_vp), _vp, _int, C.POINTER(scar_layout), _vp]),
+    "scar_ckpt_set_norm": (_int, [_vp, _int, _vp]),
     "scar_ckpt_block_scores": (_int, [_vp]),
     "scar_ckpt_priority_save": (_int, [_vp, _dbl, C.POINTER(scar_save_info)]),
     "scar_ckpt_priority_save_k": (_int, [_vp, _u64, C.POINTER(scar_save_info)]),
@@ -153,6 +155,11 @@ def scar_ckpt_init(d_x, dtype: int, layout: scar_layout, cuda_stream: int = 0) -
     _check(load_library().scar_ckpt_init(C.byref(ctx), _addr(d_x), dtype, C.byref(layout), cuda_stream or None),
            "scar_ckpt_init")
     return ctx.value
+
+
+def scar_ckpt_set_norm(ctx: int, norm: int, h_block_weights: Optional[np.ndarray] = None) -> None:
+    w = None if h_block_weights is None else np.ascontiguousarray(h_block_weights, dtype=np.float32)
+    _check(load_library().scar_ckpt_set_norm(ctx, norm, _addr(w)), "scar_ckpt_set_norm")
 
 
 def scar_ckpt_block_scores(ctx: int) -> None:
@@ -396,6 +403,11 @@ class ScarCheckpoint:
         return out
 
     # calls -------------------------------------------------------------------
+    def set_norm(self, norm: int, block_weights: Optional[np.ndarray] = None):
+        if block_weights is not None:
+            assert len(block_weights) == self.n_blocks
+        scar_ckpt_set_norm(self.ctx, norm, block_weights)
+
     def block_scores(self):
         scar_ckpt_block_scores(self.ctx)
 

@@ -18,12 +18,19 @@ namespace scar {
 
 constexpr int kThreads = 256;
 
-template <typename T> struct Elem;
+// Distance of one block: NORM 0 is the default of the element type (squared l2
+// for float32, l1 for int32); NORM 1 is the l1 distance of float32 data, which
+// with per-block weights gives the length-scaled total variation that Appendix C
+// uses for topic distributions.
+constexpr int kNormDefault = 0;
+constexpr int kNormL1 = 1;
+
+template <typename T, int NORM = kNormDefault> struct Elem;
 
 // float32 elements: squared l2 distance.  Inner chains are fp32 (at most 64
 // vectors per accumulator between flushes), the outer sum and the cross-lane
 // reduction are fp64, so long blocks do not lose accuracy.
-template <> struct Elem<float> {
+template <> struct Elem<float, kNormDefault> {
     using vec_t = float4;
     using wide_t = double;   // what a group reduces to
     using score_t = float;   // what is stored per block
@@ -39,8 +46,22 @@ template <> struct Elem<float> {
     static constexpr bool kFlush = true;
 };
 
+// float32 elements, l1 distance: same accumulation scheme with |x - z| in place of (x - z)^2.
+template <> struct Elem<float, kNormL1> {
+    using vec_t = float4;
+    using wide_t = double;
+    using score_t = float;
+    using acc_t = float;
+    static __device__ __forceinline__ void add(acc_t &a, float x, float z) { a += fabsf(x - z); }
+    static __device__ __forceinline__ void addu(acc_t &a, float x, float z) { add(a, x, z); }
+    static __device__ __forceinline__ void addu(acc_t &a, const vec_t &x, const vec_t &z) {
+        add(a, x.x, z.x); add(a, x.y, z.y); add(a, x.z, z.z); add(a, x.w, z.w);
+    }
+    static constexpr bool kFlush = true;
+};
+
 // int32 elements: integer l1 distance, exact in 64 bits (|x - z| < 2^32).
-template <> struct Elem<int> {
+template <> struct Elem<int, kNormDefault> {
     using vec_t = int4;
     using wide_t = unsigned long long;
     using score_t = unsigned long long;
@@ -95,10 +116,10 @@ __device__ __forceinline__ void load_batch(const U *__restrict__ xs, const U *__
 // in-place restore).  Accumulator slot j always takes unit lane + (4i + j) * G,
 // with or without WRITE, so the score pass and the recovery pass produce
 // bit-identical per-block sums.
-template <typename T, int G, bool VEC, bool WRITE>
-__device__ __forceinline__ typename Elem<T>::wide_t block_distance(T *__restrict__ x, const T *__restrict__ z,
-                                                                   uint64_t beg, uint64_t len, int lane) {
-    using E = Elem<T>;
+template <typename T, int NORM, int G, bool VEC, bool WRITE>
+__device__ __forceinline__ typename Elem<T, NORM>::wide_t block_distance(T *__restrict__ x, const T *__restrict__ z,
+                                                                         uint64_t beg, uint64_t len, int lane) {
+    using E = Elem<T, NORM>;
     using U = typename std::conditional<VEC, typename E::vec_t, T>::type;
     using acc_t = typename E::acc_t;
     using wide_t = typename E::wide_t;
@@ -169,19 +190,30 @@ __device__ __forceinline__ typename Elem<T>::wide_t block_distance(T *__restrict
 
 struct SelState;  // select.cuh
 
-template <typename T, int G, bool VEC>
+// Block total -> stored score, times the block's weight when the caller set
+// weights (float data only; Appendix C: a positive combination of block norms
+// is still a norm).
+template <typename E>
+__device__ __forceinline__ typename E::score_t weighted(typename E::wide_t s, const float *__restrict__ weight,
+                                                        uint64_t b) {
+    if (std::is_same<typename E::wide_t, double>::value && weight) s = (typename E::wide_t)((double)s * (double)weight[b]);
+    return (typename E::score_t)s;
+}
+
+template <typename T, int NORM, int G, bool VEC>
 __global__ void __launch_bounds__(kThreads)
-k_block_scores(const T *__restrict__ x, const T *__restrict__ z, Geom g, typename Elem<T>::score_t *__restrict__ score,
-               unsigned long long *key_or, unsigned *hist0, int hist0_len) {
-    using E = Elem<T>;
+k_block_scores(const T *__restrict__ x, const T *__restrict__ z, Geom g, const float *__restrict__ weight,
+               typename Elem<T, NORM>::score_t *__restrict__ score, unsigned long long *key_or, unsigned *hist0,
+               int hist0_len) {
+    using E = Elem<T, NORM>;
     const int lane = threadIdx.x & (G - 1);
     const uint64_t grp = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
     const bool valid = grp < g.n_blocks;
     uint64_t beg = 0, len = 0;
     if (valid) g.range((uint32_t)grp, beg, len);
-    typename E::wide_t s = block_distance<T, G, VEC, false>(const_cast<T *>(x), z, beg, len, lane);
+    typename E::wide_t s = block_distance<T, NORM, G, VEC, false>(const_cast<T *>(x), z, beg, len, lane);
     if (valid && lane == 0) {
-        typename E::score_t sc = (typename E::score_t)s;
+        typename E::score_t sc = weighted<E>(s, weight, grp);
         score[grp] = sc;
         if (sizeof(typename E::score_t) == 8) {
             // Remember which key bits occur at all, so that radix passes over
@@ -198,11 +230,11 @@ k_block_scores(const T *__restrict__ x, const T *__restrict__ z, Geom g, typenam
 
 // ---- a4 / a5: per-block perturbation over the lost set, optional restore ---
 
-template <typename T, int G, bool VEC, bool WRITE>
+template <typename T, int NORM, int G, bool VEC, bool WRITE>
 __global__ void __launch_bounds__(kThreads)
-k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S,
-                 typename Elem<T>::score_t *__restrict__ part) {
-    using E = Elem<T>;
+k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S, const float *__restrict__ weight,
+                 typename Elem<T, NORM>::score_t *__restrict__ part) {
+    using E = Elem<T, NORM>;
     const int lane = threadIdx.x & (G - 1);
     if (G < 32 && S.mode == 2) {
         // Per-block mask with several blocks per warp: a warp takes 32 consecutive
@@ -223,8 +255,8 @@ k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S,
                 b = (uint32_t)(b0 + __fns(bal, 0, t + 1));
                 g.range(b, beg, len);
             }
-            typename E::wide_t s = block_distance<T, G, VEC, WRITE>(x, z, beg, len, lane);
-            if (valid && lane == 0) part[b] = (typename E::score_t)s;
+            typename E::wide_t s = block_distance<T, NORM, G, VEC, WRITE>(x, z, beg, len, lane);
+            if (valid && lane == 0) part[b] = weighted<E>(s, weight, b);
         }
         return;
     }
@@ -233,8 +265,8 @@ k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S,
     const bool valid = S.block_of(w, b);
     uint64_t beg = 0, len = 0;
     if (valid) g.range(b, beg, len);
-    typename E::wide_t s = block_distance<T, G, VEC, WRITE>(x, z, beg, len, lane);
-    if (valid && lane == 0) part[b] = (typename E::score_t)s;
+    typename E::wide_t s = block_distance<T, NORM, G, VEC, WRITE>(x, z, beg, len, lane);
+    if (valid && lane == 0) part[b] = weighted<E>(s, weight, b);
 }
 
 // Lost shards as a per-block mask, for lost sets with more runs than LostSet holds.
@@ -276,7 +308,7 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 k_reduce_partials(const typename Elem<T>::score_t *__restrict__ part, Geom g, LostSet S, double *tile_sum,
                   unsigned long long *tile_l1, unsigned long long *tile_blocks, unsigned long long *tile_elems,
-                  unsigned *ticket, NormInfoDev *out) {
+                  unsigned *ticket, NormInfoDev *out, bool take_sqrt) {
     __shared__ double shd[kThreads / 32];
     __shared__ unsigned long long shu[kThreads / 32];
     __shared__ bool is_last;
@@ -327,7 +359,7 @@ k_reduce_partials(const typename Elem<T>::score_t *__restrict__ part, Geom g, Lo
     nb = cta_sum<unsigned long long>(nb, shu);
     ne = cta_sum<unsigned long long>(ne, shu);
     if (threadIdx.x == 0) {
-        out->l2 = sqrt(fs);
+        out->l2 = take_sqrt ? sqrt(fs) : fs;  // l2 norms sum squares; l1 / weighted-l1 norms sum as they are
         out->l1 = is;
         out->lost_blocks = nb;
         out->lost_elems = ne;

@@ -59,6 +59,9 @@ struct scar_ctx {
     void *score = nullptr;  // float[B] or uint64[B]
     void *part = nullptr;   // per-block perturbation partials, same type as score
     uint64_t *d_boff = nullptr;
+    int norm = SCAR_NORM_DEFAULT;
+    float *d_weight = nullptr;  // per-block weights of the norm, or nullptr
+    float *d_weight_buf = nullptr;
     uint8_t *d_shard_mask = nullptr;
     uint8_t *d_block_mask = nullptr;  // only used when a shard mask has too many runs
     SelState *st = nullptr;
@@ -198,17 +201,23 @@ void record(scar_ctx *c, int i) {
 }
 
 // a1
-template <typename T> void launch_scores(scar_ctx *c) {
-    using S = typename Elem<T>::score_t;
-    if (c->g.n_blocks == 0) return;
+template <typename T, int NORM> void launch_scores_as(scar_ctx *c) {
+    using S = typename Elem<T, NORM>::score_t;
     dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
         constexpr int G = decltype(gl)::value;
         constexpr bool VEC = decltype(vec)::value;
-        k_block_scores<T, G, VEC><<<grid_for_groups(c->g.n_blocks, G), kThreads, 0, c->stream>>>(
-            static_cast<const T *>(c->x), static_cast<const T *>(c->z), c->g, static_cast<S *>(c->score),
+        k_block_scores<T, NORM, G, VEC><<<grid_for_groups(c->g.n_blocks, G), kThreads, 0, c->stream>>>(
+            static_cast<const T *>(c->x), static_cast<const T *>(c->z), c->g, c->d_weight, static_cast<S *>(c->score),
             &c->st->key_or, c->st->hist[0], kHistBins);
     });
     ++c->launches;
+}
+
+void launch_scores(scar_ctx *c) {
+    if (c->g.n_blocks == 0) return;
+    if (c->dt == SCAR_I32) launch_scores_as<int, kNormDefault>(c);
+    else if (c->norm == SCAR_NORM_L1) launch_scores_as<float, kNormL1>(c);
+    else launch_scores_as<float, kNormDefault>(c);
 }
 
 // a2: one cooperative launch (all CTAs resident, so its grid-wide barriers cannot deadlock)
@@ -255,8 +264,8 @@ void launch_pack(scar_ctx *c, uint64_t k) {
 }
 
 // a4 / a5
-template <typename T> void launch_recover(scar_ctx *c, const LostSet &S, bool write) {
-    using Sc = typename Elem<T>::score_t;
+template <typename T, int NORM> void launch_recover_as(scar_ctx *c, const LostSet &S, bool write) {
+    using Sc = typename Elem<T, NORM>::score_t;
     if (S.n_work > 0) {
         dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
             constexpr int G = decltype(gl)::value;
@@ -265,11 +274,13 @@ template <typename T> void launch_recover(scar_ctx *c, const LostSet &S, bool wr
             const unsigned grid = (G < 32 && S.mode == 2) ? (unsigned)((S.n_work + kThreads - 1) / kThreads)
                                                           : grid_for_groups(S.n_work, G);
             if (write)
-                k_recover_blocks<T, G, VEC, true><<<grid, kThreads, 0, c->stream>>>(
-                    static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, static_cast<Sc *>(c->part));
+                k_recover_blocks<T, NORM, G, VEC, true><<<grid, kThreads, 0, c->stream>>>(
+                    static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, c->d_weight,
+                    static_cast<Sc *>(c->part));
             else
-                k_recover_blocks<T, G, VEC, false><<<grid, kThreads, 0, c->stream>>>(
-                    static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, static_cast<Sc *>(c->part));
+                k_recover_blocks<T, NORM, G, VEC, false><<<grid, kThreads, 0, c->stream>>>(
+                    static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, c->d_weight,
+                    static_cast<Sc *>(c->part));
         });
         ++c->launches;
     }
@@ -278,9 +289,15 @@ template <typename T> void launch_recover(scar_ctx *c, const LostSet &S, bool wr
     if (tiles == 0) tiles = 1;
     k_reduce_partials<T><<<(unsigned)tiles, kThreads, 0, c->stream>>>(
         static_cast<const Sc *>(c->part), c->g, S, c->rt_sum, c->rt_l1, c->rt_blocks, c->rt_elems,
-        &c->st->ticket_reduce, c->d_norm);
+        &c->st->ticket_reduce, c->d_norm, NORM == kNormDefault);
     ++c->launches;
     record(c, 5);
+}
+
+void launch_recover(scar_ctx *c, const LostSet &S, bool write) {
+    if (c->dt == SCAR_I32) launch_recover_as<int, kNormDefault>(c, S, write);
+    else if (c->norm == SCAR_NORM_L1) launch_recover_as<float, kNormL1>(c, S, write);
+    else launch_recover_as<float, kNormDefault>(c, S, write);
 }
 
 int copy_elems(scar_ctx *c, void *dst, const void *src, uint64_t n) {
@@ -353,8 +370,7 @@ int enqueue_save(scar_ctx *c, uint64_t k) {
         c->have_save = true;
         return SCAR_OK;
     }
-    if (c->dt == SCAR_F32) launch_scores<float>(c);
-    else launch_scores<int>(c);
+    launch_scores(c);
     record(c, 1);
     const int rc_sel = c->dt == SCAR_F32
                            ? launch_select<float>(c, static_cast<const float *>(c->score), k)
@@ -413,8 +429,7 @@ int enqueue_recover(scar_ctx *c, const LostSet &S, bool write) {
         c->have_norm = true;
         return SCAR_OK;
     }
-    if (c->dt == SCAR_F32) launch_recover<float>(c, S, write);
-    else launch_recover<int>(c, S, write);
+    launch_recover(c, S, write);
     CU_TRY(cudaGetLastError());
     c->have_norm = true;
     return SCAR_OK;
@@ -598,8 +613,7 @@ int scar_ckpt_block_scores(scar_ctx *c) {
     if (rc != SCAR_OK) return rc;
     c->last_call = 3;
     record(c, 0);
-    if (c->dt == SCAR_F32) launch_scores<float>(c);
-    else launch_scores<int>(c);
+    launch_scores(c);
     record(c, 1);
     CU_TRY(cudaGetLastError());
     return SCAR_OK;
@@ -756,6 +770,28 @@ int scar_recover_partial_host(scar_ctx *c, void *h_x, const uint8_t *h_lost_shar
     for (size_t i = 0; i < lo.size(); ++i)
         CU_TRY(cudaMemcpyAsync(hx + lo[i] * 4, dx + lo[i] * 4, (hi[i] - lo[i]) * 4, cudaMemcpyDeviceToHost, c->stream));
     return fetch_norm(c, out);
+}
+
+int scar_ckpt_set_norm(scar_ctx *c, scar_norm norm, const float *h_block_weights) {
+    if (!c || (norm != SCAR_NORM_DEFAULT && norm != SCAR_NORM_L1)) return SCAR_ERR_INVALID_ARG;
+    if (c->dt == SCAR_I32 && h_block_weights) return SCAR_ERR_INVALID_ARG;  // integer scores stay exact integers
+    const uint64_t B = c->g.n_blocks;
+    if (h_block_weights)
+        for (uint64_t b = 0; b < B; ++b)
+            if (!(h_block_weights[b] >= 0.0f) || std::isinf(h_block_weights[b])) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    if (h_block_weights && B) {
+        if (!c->d_weight_buf && (rc = dev_alloc(c, &c->d_weight_buf, B * 4)) != SCAR_OK) return rc;
+        // pageable source: the copy has read h_block_weights by the time this returns
+        CU_TRY(cudaMemcpyAsync(c->d_weight_buf, h_block_weights, B * 4, cudaMemcpyHostToDevice, c->stream));
+        CU_TRY(cudaStreamSynchronize(c->stream));
+        c->d_weight = c->d_weight_buf;
+    } else {
+        c->d_weight = nullptr;
+    }
+    c->norm = norm;
+    return SCAR_OK;
 }
 
 int scar_ckpt_drain_init(scar_ctx *c, uint64_t max_k, uint64_t max_payload_elems) {

@@ -84,7 +84,7 @@ int run_static(const void *d_x, const void *d_z, const Geom &g, const LostSet &S
     T *x = static_cast<T *>(const_cast<void *>(d_x));  // the read-only instantiation never stores
     const T *z = static_cast<const T *>(d_z);
 #define SCAR_STATIC_LAUNCH(G_, VEC_) \
-    k_recover_blocks<T, G_, VEC_, false><<<grid, kThreads, 0, stream>>>(x, z, g, S, part)
+    k_recover_blocks<T, kNormDefault, G_, VEC_, false><<<grid, kThreads, 0, stream>>>(x, z, g, S, nullptr, part)
     if (g.vec_ok) {
         if (G == 4) SCAR_STATIC_LAUNCH(4, true);
         else if (G == 8) SCAR_STATIC_LAUNCH(8, true);
@@ -99,7 +99,7 @@ int run_static(const void *d_x, const void *d_z, const Geom &g, const LostSet &S
 #undef SCAR_STATIC_LAUNCH
     const unsigned tiles = (unsigned)((g.n_blocks + kReduceTile - 1) / kReduceTile);
     k_reduce_partials<T><<<tiles, kThreads, 0, stream>>>(part, g, S, tile_sum, tile_l1, tile_blocks, tile_elems, ticket,
-                                                        reinterpret_cast<NormInfoDev *>(d_out));
+                                                        reinterpret_cast<NormInfoDev *>(d_out), true);
     return cudaGetLastError() == cudaSuccess ? SCAR_OK : SCAR_ERR_CUDA;
 }
 

@@ -491,6 +491,111 @@ def test_theorem_4_2_partition_identity_and_expectation():
     assert stderr < 0.05 * p * full, "the check has power"
 
 
+# ---- weighted norms and total variation (Appendix C) -------------------------------------------
+
+
+def test_l1_scores_of_distributions_are_twice_the_total_variation():
+    """TV(p, q) = max over events A of |p(A) - q(A)| (brute force over all subsets) = (1/2) sum |p - q|."""
+    r = rng(40)
+    k, nb = 7, 12
+    p = r.dirichlet(np.ones(k), size=nb).astype(np.float32)
+    q = r.dirichlet(np.ones(k), size=nb).astype(np.float32)
+    boff = (np.arange(nb + 1, dtype=np.uint64) * k)
+    l1 = oracle.block_scores_norm(p.ravel(), q.ravel(), boff, "l1")
+    for b in range(nb):
+        d = p[b].astype(np.float64) - q[b].astype(np.float64)
+        tv = max(abs(sum(d[i] for i in range(k) if mask >> i & 1)) for mask in range(1 << k))
+        # float32 rows do not sum to exactly 1; the two sides differ by at most half that defect
+        assert abs(0.5 * l1[b] - tv) <= 0.5 * abs(d.sum()) + 1e-15
+
+
+def test_length_scaled_tv_of_count_rows_is_half_their_l1():
+    """Appendix C: scaling the total variation of a document's topic distribution by the document's length removes
+    the bias towards short documents: moving one token costs the same in every document."""
+    r = rng(41)
+    k = 20
+    lengths = np.array([5, 50, 500, 5000])
+    counts = np.stack([r.multinomial(n, np.ones(k) / k) for n in lengths])
+    moved = counts.copy()
+    for d in range(lengths.size):  # re-sample one token: one count down, another up
+        src = int(np.flatnonzero(moved[d])[0])
+        moved[d, src] -= 1
+        moved[d, (src + 1) % k] += 1
+    p = (counts / lengths[:, None]).astype(np.float32).ravel()
+    q = (moved / lengths[:, None]).astype(np.float32).ravel()
+    boff = (np.arange(lengths.size + 1, dtype=np.uint64) * k)
+    plain = 0.5 * oracle.block_scores_norm(p, q, boff, "l1")
+    scaled = oracle.block_scores_norm(p, q, boff, "l1", weights=lengths / 2.0)
+    assert plain[0] > 100 * plain[3]  # unweighted: the short document dominates
+    np.testing.assert_allclose(scaled, 1.0, rtol=1e-5)  # scaled: one token each
+    # and it equals half the l1 of the count rows themselves (the integer path)
+    ints = oracle.block_scores(counts.astype(np.int32).ravel(), moved.astype(np.int32).ravel(), boff)
+    np.testing.assert_allclose(scaled, ints / 2.0, rtol=1e-5)
+
+
+def test_weighted_scores_bruteforce_and_special_weights():
+    x, z, boff = small_case(42, np.float32, nb=40)
+    nb = boff.size - 1
+    ids = block_ids(boff)
+    w = rng(43).uniform(0, 3, nb)
+    for norm in ("l2", "l1"):
+        got = oracle.block_scores_norm(x, z, boff, norm, w)
+        for b in range(nb):
+            d = x[ids == b].astype(np.float64) - z[ids == b].astype(np.float64)
+            want = w[b] * (math.fsum(d * d) if norm == "l2" else math.fsum(np.abs(d)))
+            assert math.isclose(got[b], want, rel_tol=1e-13, abs_tol=0.0) or got[b] == want == 0.0
+        np.testing.assert_array_equal(oracle.block_scores_norm(x, z, boff, norm, np.ones(nb)),
+                                      oracle.block_scores_norm(x, z, boff, norm))
+        assert not oracle.block_scores_norm(x, z, boff, norm, np.zeros(nb)).any()
+    np.testing.assert_array_equal(oracle.block_scores_norm(x, z, boff, "l2"), oracle.block_scores(x, z, boff))
+
+
+def test_weighted_perturbation_is_a_norm_and_matches_the_plain_one():
+    x, z, boff = small_case(44, np.float32, nb=50)
+    nb = boff.size - 1
+    r = rng(45)
+    w = r.uniform(0.1, 4, nb)
+    lost = (r.random(nb) < 0.4).astype(np.uint8)
+    plain = oracle.perturbation_norm(x, z, boff, lost)
+    same = oracle.perturbation_norm_weighted(x, z, boff, lost, "l2")
+    assert math.isclose(same.l2, plain.l2, rel_tol=1e-13) and same.lost_blocks == plain.lost_blocks
+    assert same.lost_elems == plain.lost_elems
+    for norm in ("l2", "l1"):
+        full = oracle.perturbation_norm_weighted(x, z, boff, None, norm, w).l2
+        part = oracle.perturbation_norm_weighted(x, z, boff, lost, norm, w).l2
+        assert 0 < part <= full  # Theorem 4.1 carries over: disjoint supports
+        # homogeneity: scaling the difference by 3 scales the norm by 3
+        x3 = (z.astype(np.float64) + 3.0 * (x.astype(np.float64) - z.astype(np.float64)))
+        d1 = oracle.block_scores_norm(x, z, boff, norm, w)
+        # triangle inequality on random splits of the difference: ||a + b|| <= ||a|| + ||b||
+        a = (r.random(x.size) * (x - z)).astype(np.float32)
+        b = ((x - z) - a).astype(np.float32)
+        zero = np.zeros_like(x)
+        na = oracle.perturbation_norm_weighted(a, zero, boff, None, norm, w).l2
+        nb_ = oracle.perturbation_norm_weighted(b, zero, boff, None, norm, w).l2
+        nab = oracle.perturbation_norm_weighted((a + b).astype(np.float32), zero, boff, None, norm, w).l2
+        assert nab <= (na + nb_) * (1 + 1e-12)
+        n3 = oracle.perturbation_norm_weighted((3 * (a + b)).astype(np.float32), zero, boff, None, norm, w).l2
+        assert math.isclose(n3, 3 * nab, rel_tol=1e-6)
+        del x3, d1
+
+
+def test_weights_change_what_a_prioritized_save_takes():
+    # one heavily weighted block with a small change outranks unweighted blocks with larger changes
+    nb, blk = 8, 4
+    z = np.zeros(nb * blk, dtype=np.float32)
+    x = z.copy()
+    x[0:4] = 0.1      # block 0: small change
+    x[4:8] = 1.0      # block 1: large change
+    x[8:12] = 0.5     # block 2
+    boff = (np.arange(nb + 1, dtype=np.uint64) * blk)
+    assert oracle.save_norm(x, z, boff, 1, "l1").sel.tolist() == [1]
+    w = np.ones(nb)
+    w[0] = 100.0
+    assert oracle.save_norm(x, z, boff, 1, "l1", w).sel.tolist() == [0]
+    assert oracle.save_norm(x, z, boff, 2, "l2", w).sel.tolist() == [0, 1]  # 100 * 0.04 = 4 > 4 * 0.25 = 1
+
+
 # ---- baseline selectors (Section 5.4) ---------------------------------------------------
 
 
