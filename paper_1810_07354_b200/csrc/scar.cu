@@ -14,6 +14,7 @@
 
 #include "block_pass.cuh"
 #include "pack.cuh"
+#include "segments.cuh"
 #include "select.cuh"
 
 using namespace scar;
@@ -59,6 +60,13 @@ struct scar_ctx {
     void *score = nullptr;  // float[B] or uint64[B]
     void *part = nullptr;   // per-block perturbation partials, same type as score
     uint64_t *d_boff = nullptr;
+    // segment mode (layouts with very long blocks)
+    bool seg_mode = false;
+    Segs segs{};
+    void *seg_part = nullptr;      // double[n_segs] or uint64[n_segs]
+    uint32_t *selpos = nullptr;    // B: position in the id list, 0xffffffff when not selected
+    uint32_t *wide_blocks = nullptr;  // blocks with more than kWideSegs segments
+    unsigned n_wide_blocks = 0;
     int norm = SCAR_NORM_DEFAULT;
     float *d_weight = nullptr;  // per-block weights of the norm, or nullptr
     float *d_weight_buf = nullptr;
@@ -213,8 +221,46 @@ template <typename T, int NORM> void launch_scores_as(scar_ctx *c) {
     ++c->launches;
 }
 
+unsigned grid_for_warps(uint64_t n_warps) { return (unsigned)((n_warps + kThreads / 32 - 1) / (kThreads / 32)); }
+
+// Segment sums -> block totals: one warp per block, plus one CTA per block that has very many segments.
+template <typename T, int NORM>
+void launch_combine(scar_ctx *c, const typename Elem<T, NORM>::wide_t *sp, const uint8_t *mask,
+                    typename Elem<T, NORM>::score_t *out, unsigned long long *key_or, unsigned *hist0, int hist0_len) {
+    k_combine_segments<T, NORM, false><<<grid_for_warps(c->g.n_blocks), kThreads, 0, c->stream>>>(
+        c->segs, c->g.n_blocks, nullptr, sp, c->d_weight, mask, out, key_or, hist0, hist0_len);
+    ++c->launches;
+    if (c->n_wide_blocks) {
+        k_combine_segments<T, NORM, true><<<c->n_wide_blocks, kThreads, 0, c->stream>>>(
+            c->segs, c->g.n_blocks, c->wide_blocks, sp, c->d_weight, mask, out, key_or, nullptr, 0);
+        ++c->launches;
+    }
+}
+
+template <typename T, int NORM> void launch_segment_scores(scar_ctx *c) {
+    using W = typename Elem<T, NORM>::wide_t;
+    using S = typename Elem<T, NORM>::score_t;
+    T *x = static_cast<T *>(c->x);
+    const T *z = static_cast<const T *>(c->z);
+    W *sp = static_cast<W *>(c->seg_part);
+    if (c->g.vec_ok)
+        k_segment_pass<T, NORM, true, false><<<grid_for_warps(c->segs.n), kThreads, 0, c->stream>>>(x, z, c->g, c->segs,
+                                                                                                 nullptr, sp);
+    else
+        k_segment_pass<T, NORM, false, false><<<grid_for_warps(c->segs.n), kThreads, 0, c->stream>>>(x, z, c->g, c->segs,
+                                                                                                  nullptr, sp);
+    launch_combine<T, NORM>(c, sp, nullptr, static_cast<S *>(c->score), &c->st->key_or, c->st->hist[0], kHistBins);
+    ++c->launches;
+}
+
 void launch_scores(scar_ctx *c) {
     if (c->g.n_blocks == 0) return;
+    if (c->seg_mode) {
+        if (c->dt == SCAR_I32) launch_segment_scores<int, kNormDefault>(c);
+        else if (c->norm == SCAR_NORM_L1) launch_segment_scores<float, kNormL1>(c);
+        else launch_segment_scores<float, kNormDefault>(c);
+        return;
+    }
     if (c->dt == SCAR_I32) launch_scores_as<int, kNormDefault>(c);
     else if (c->norm == SCAR_NORM_L1) launch_scores_as<float, kNormL1>(c);
     else launch_scores_as<float, kNormDefault>(c);
@@ -253,6 +299,21 @@ int plan_select(scar_ctx *c) {
 // a3
 void launch_pack(scar_ctx *c, uint64_t k) {
     if (k == 0) return;
+    if (c->seg_mode) {
+        cudaMemsetAsync(c->selpos, 0xff, c->g.n_blocks * 4, c->stream);
+        k_mark_selected<<<(unsigned)((k + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(c->cur.sel, c->cur.info,
+                                                                                              c->selpos);
+        const uint32_t *x = static_cast<const uint32_t *>(c->x);
+        uint32_t *z = static_cast<uint32_t *>(c->z), *pay = static_cast<uint32_t *>(c->cur.payload);
+        if (c->g.vec_ok)
+            k_pack_segments<true><<<grid_for_warps(c->segs.n), kThreads, 0, c->stream>>>(x, z, pay, c->g, c->segs,
+                                                                                       c->selpos, c->cur.poff);
+        else
+            k_pack_segments<false><<<grid_for_warps(c->segs.n), kThreads, 0, c->stream>>>(x, z, pay, c->g, c->segs,
+                                                                                        c->selpos, c->cur.poff);
+        c->launches += 2;
+        return;
+    }
     dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
         constexpr int G = decltype(gl)::value;
         constexpr bool VEC = decltype(vec)::value;
@@ -266,7 +327,24 @@ void launch_pack(scar_ctx *c, uint64_t k) {
 // a4 / a5
 template <typename T, int NORM> void launch_recover_as(scar_ctx *c, const LostSet &S, bool write) {
     using Sc = typename Elem<T, NORM>::score_t;
-    if (S.n_work > 0) {
+    if (c->seg_mode && S.n_work > 0) {
+        // S is "all blocks" (mode 0) or a per-block mask (mode 2) here: enqueue_recover turns shard runs into a mask
+        using W = typename Elem<T, NORM>::wide_t;
+        T *x = static_cast<T *>(c->x);
+        const T *z = static_cast<const T *>(c->z);
+        W *sp = static_cast<W *>(c->seg_part);
+        const uint8_t *mask = S.mode == 2 ? S.mask : nullptr;
+        const unsigned grid = grid_for_warps(c->segs.n);
+        if (c->g.vec_ok) {
+            if (write) k_segment_pass<T, NORM, true, true><<<grid, kThreads, 0, c->stream>>>(x, z, c->g, c->segs, mask, sp);
+            else k_segment_pass<T, NORM, true, false><<<grid, kThreads, 0, c->stream>>>(x, z, c->g, c->segs, mask, sp);
+        } else {
+            if (write) k_segment_pass<T, NORM, false, true><<<grid, kThreads, 0, c->stream>>>(x, z, c->g, c->segs, mask, sp);
+            else k_segment_pass<T, NORM, false, false><<<grid, kThreads, 0, c->stream>>>(x, z, c->g, c->segs, mask, sp);
+        }
+        ++c->launches;
+        launch_combine<T, NORM>(c, sp, mask, static_cast<Sc *>(c->part), nullptr, nullptr, 0);
+    } else if (S.n_work > 0) {
         dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
             constexpr int G = decltype(gl)::value;
             constexpr bool VEC = decltype(vec)::value;
@@ -479,7 +557,7 @@ int shard_set(scar_ctx *c, const uint8_t *h_lost_shards, LostSet &S) {
         S.run_start[S.n_runs] = (uint32_t)work;
     }
     S.n_work = work;
-    if (!overflow) return SCAR_OK;
+    if (!overflow && !c->seg_mode) return SCAR_OK;  // segment mode walks segments, so it always wants a block mask
     CU_TRY(cudaMemcpyAsync(c->d_shard_mask, h_lost_shards, n_sh, cudaMemcpyHostToDevice, c->stream));
     k_expand_shards<<<(unsigned)((B + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(c->g, c->d_shard_mask,
                                                                                           c->d_block_mask);
@@ -578,6 +656,52 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     A(&c->cur.info, sizeof(SaveInfoDev));
     A(&c->d_norm, sizeof(NormInfoDev));
     if (rc == SCAR_OK && layout->block_offsets) A(&c->d_boff, (B + 1) * 8);
+    // Very long blocks: cut every block into segments (see segments.cuh).  The host tables live until the
+    // stream synchronisation at the end of init.
+    std::vector<uint32_t> seg_block, wide;
+    std::vector<uint64_t> seg_beg, seg_first;
+    if (rc == SCAR_OK && c->max_block_len > 2 * kSegElems) {
+        seg_first.resize(B + 1);
+        for (uint64_t b = 0; b < B; ++b) {
+            uint64_t beg, len;
+            if (layout->block_offsets) {
+                beg = layout->block_offsets[b];
+                len = layout->block_offsets[b + 1] - beg;
+            } else {
+                const uint64_t row = b / g.blocks_per_row, j = b % g.blocks_per_row, o = j * g.block_elems;
+                beg = row * g.row_len + o;
+                len = g.row_len - o < g.block_elems ? g.row_len - o : g.block_elems;
+            }
+            seg_first[b] = seg_block.size();
+            for (uint64_t o = 0; o < len; o += kSegElems) {
+                seg_block.push_back((uint32_t)b);
+                seg_beg.push_back(beg + o);
+            }
+        }
+        seg_first[B] = seg_block.size();
+        for (uint64_t b = 0; b < B; ++b)
+            if (seg_first[b + 1] - seg_first[b] > kWideSegs) wide.push_back((uint32_t)b);
+        const uint64_t ns = seg_block.size();
+        uint32_t *d_sb = nullptr;
+        uint64_t *d_sbeg = nullptr, *d_sfirst = nullptr;
+        A(&d_sb, ns * 4);
+        A(&d_sbeg, ns * 8);
+        A(&d_sfirst, (B + 1) * 8);
+        A(&c->seg_part, ns * 8);
+        A(&c->selpos, B * 4);
+        A(&c->wide_blocks, wide.size() * 4);
+        c->n_wide_blocks = (unsigned)wide.size();
+        if (rc == SCAR_OK && !wide.empty() &&
+            cudaMemcpyAsync(c->wide_blocks, wide.data(), wide.size() * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+            rc = SCAR_ERR_CUDA;
+        if (rc == SCAR_OK &&
+            (cudaMemcpyAsync(d_sb, seg_block.data(), ns * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
+             cudaMemcpyAsync(d_sbeg, seg_beg.data(), ns * 8, cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
+             cudaMemcpyAsync(d_sfirst, seg_first.data(), (B + 1) * 8, cudaMemcpyHostToDevice, c->stream) != cudaSuccess))
+            rc = SCAR_ERR_CUDA;
+        c->segs = Segs{d_sb, d_sbeg, d_sfirst, ns};
+        c->seg_mode = rc == SCAR_OK;
+    }
     if (rc == SCAR_OK && (cudaMallocHost(&c->h_save, sizeof(SaveInfoDev)) != cudaSuccess ||
                           cudaMallocHost(&c->h_norm, sizeof(NormInfoDev)) != cudaSuccess))
         rc = SCAR_ERR_ALLOC;

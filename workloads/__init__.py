@@ -14,4 +14,6 @@ from .configs import (  # noqa: F401
     make_workload,
     block_offsets,
     shard_block_ranges,
+    bylayer_offsets,
+    make_cnn_bylayer,
 )

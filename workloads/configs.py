@@ -228,6 +228,33 @@ def make_cnn_device(n_elems: int = 1 << 30, block_elems: int = 4096, seed: int =
     return geom, z, x, lost
 
 
+def bylayer_offsets(scale: int = 1, pad_to: int = 1) -> np.ndarray:
+    """Block offsets of a network checkpointed by layer (Section 5.1, by-layer partitioning): weight and bias of two
+    convolutions and three fully connected layers, each tensor one block, so block lengths span five orders of
+    magnitude.  ``scale`` widens every layer; ``pad_to`` rounds lengths up (4 keeps every block 16-byte aligned)."""
+    c1, c2, f1, f2, classes = 32 * scale, 64 * scale, 1024 * scale, 512 * scale, 10
+    lens = [25 * 1 * c1, c1, 25 * c1 * c2, c2, 49 * c2 * f1, f1, f1 * f2, f2, f2 * classes, classes]
+    lens = [-(-n // pad_to) * pad_to for n in lens]
+    return np.concatenate([[0], np.cumsum(lens)]).astype(np.uint64)
+
+
+def make_cnn_bylayer(scale: int = 1, pad_to: int = 1, dtype: str = "f32", seed: int = 5):
+    """Returns ``(boff, z, x)`` for the by-layer layout: per-layer change scale ``1 + Pareto(1.5)`` times
+    N(0, 1e-3) noise around N(0, 5e-2) weights (float32), or Poisson counts with small integer changes (int32)."""
+    rng = _rng(seed)
+    boff = bylayer_offsets(scale, pad_to)
+    lens = np.diff(boff.astype(np.int64))
+    n = int(boff[-1])
+    if dtype == "f32":
+        z = (rng.standard_normal(n, dtype=np.float32) * np.float32(5e-2)).astype(np.float32)
+        a = (1.0 + rng.pareto(1.5, size=lens.size)).astype(np.float32)
+        x = (z + rng.standard_normal(n, dtype=np.float32) * np.float32(1e-3) * np.repeat(a, lens)).astype(np.float32)
+    else:
+        z = rng.poisson(3.0, size=n).astype(np.int32)
+        x = np.maximum(z + rng.integers(-2, 3, size=n), 0).astype(np.int32)
+    return boff, z, x
+
+
 CONFIGS = {
     "tiny": make_tiny,
     "mlr": make_mlr,
