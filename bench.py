@@ -450,10 +450,122 @@ def run_gpu(args):
         else:
             lb = lost_blocks
         line["cpu_baseline"] = cpu_baseline(x0, z0, geom, lb, r_sweep)
+    if world == 1 and not args.no_extras:
+        line["extras"] = run_extras(api, ck, x, x0, z_lib, z0, geom, r_sweep, flush, dev,
+                                    with_bylayer=args.workload == "cnn" and n >= (1 << 28))
     print(json.dumps(line))
     barrier()
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_extras(api, ck, x, x0, z_lib, z0, geom, r_sweep, flush, dev, with_bylayer):
+    """Measurements beside the headline step, outside its timed region: the two baseline selectors
+    (Section 5.4), the asynchronous drain (Section 4.3) and a by-layer layout with very unequal blocks
+    (Section 5.1).  Device times from CUDA events / the library's phase events; the drain is wall-clock because
+    it ends on the host."""
+    import torch
+
+    from workloads import bylayer_offsets
+
+    n, nb = x.numel(), ck.n_blocks
+    r = r_sweep[min(1, len(r_sweep) - 1)]
+    k = max(1, int(r * nb + 0.5))
+    out = {"r": r, "k": k}
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+
+    def timed(fn, reps=10):
+        ts = []
+        for _ in range(reps + 2):
+            z_lib.copy_(z0)
+            flush.zero_()
+            a, b = ev(), ev()
+            a.record()
+            fn()
+            b.record()
+            b.synchronize()
+            ts.append(a.elapsed_time(b))
+        return float(np.median(ts[2:]))
+
+    pri = torch.randint(0, 2**31 - 1, (nb,), device=dev, dtype=torch.int32)
+    info = ck.save_round(k)
+    pay = int(info.payload_elems)
+    for name, fn in (("priority", lambda: ck.priority_save_k(k, sync=False)),
+                     ("round", lambda: ck.save_round(k, sync=False)),
+                     ("random", lambda: ck.save_random(k, pri, sync=False))):
+        ms = timed(fn)
+        moved = 3 * pay * ELEM + (2 * n * ELEM if name == "priority" else 0)
+        out[name] = {"save_ms": ms, "algorithmic_gbs": moved / ms / 1e6}
+
+    # ---- asynchronous drain: saves keep running on the context's stream while the previous payload goes to
+    # pinned host memory on the drain stream
+    block_len = geom.block_elems if geom.block_elems else n
+    ck.drain_init(k, min(n, k * min(block_len, geom.row_len)))
+    dump_ms, tickets, n_saves = [], [], 6
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(n_saves):
+        z_lib.copy_(z0)
+        a, b = ev(), ev()
+        a.record()
+        ck.priority_save_k(k, sync=False)
+        b.record()
+        tickets.append((ck.drain_enqueue(), a, b))
+        if len(tickets) >= 2:  # two slots: take the older payload off the host side before the next save
+            t_old, a_old, b_old = tickets.pop(0)
+            ck.drain_wait(t_old)
+            ck.drain_release(t_old)
+            dump_ms.append(a_old.elapsed_time(b_old))
+    t_old, a_old, b_old = tickets.pop(0)
+    view = ck.drain_wait(t_old)
+    drained = int(view["info"].payload_elems) * ELEM + int(view["info"].k) * 12 + 40
+    ck.drain_release(t_old)
+    dump_ms.append(a_old.elapsed_time(b_old))
+    wall_ms = 1e3 * (time.perf_counter() - t0) / n_saves
+    # one save + drain with nothing else in flight, for the copy rate alone
+    z_lib.copy_(z0)
+    ck.priority_save_k(k, sync=False)
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    t = ck.drain_enqueue()
+    ck.drain_wait(t)
+    copy_ms = 1e3 * (time.perf_counter() - t1)
+    ck.drain_release(t)
+    out["drain"] = {"t_dump_ms": float(np.median(dump_ms)), "pipelined_ms_per_save": wall_ms,
+                    "drain_alone_ms": copy_ms, "drained_bytes": drained, "drain_gbs": drained / copy_ms / 1e6,
+                    "note": "t_dump = score + select + pack + cache refresh on the context's stream while the "
+                            "previous payload is copied out; pipelined = wall-clock per save of 6 back-to-back "
+                            "save + drain rounds (PCIe-bound)"}
+
+    # ---- by-layer layout: 10 tensors from 12 to 8.2e8 elements, cut into segments by the library
+    if with_bylayer:
+        boff = bylayer_offsets(scale=16, pad_to=4)
+        nl = int(boff[-1])
+        g = torch.Generator(device=dev).manual_seed(11)
+        zl = torch.randn(nl, device=dev, generator=g) * 5e-2
+        xl = zl + torch.randn(nl, device=dev, generator=g) * 1e-3
+        cl = api.ScarCheckpoint(xl, n_shards=5, block_offsets=boff)
+        api.scar_ckpt_profile(cl.ctx, True)
+        rows = []
+        for _ in range(5):
+            cl.load(zl)
+            flush.zero_()
+            cl.priority_save_k(5, sync=False)
+            ph = api.scar_ckpt_profile_read(cl.ctx)
+            pe = int(api.scar_ckpt_last_info(cl.ctx, True, False)[0].payload_elems)
+            flush.zero_()
+            cl.recover_partial(np.array([0, 0, 1, 0, 0], dtype=np.uint8), sync=False)
+            rp = api.scar_ckpt_profile_read(cl.ctx)
+            le = int(api.scar_ckpt_last_info(cl.ctx, False, True)[1].lost_elems)
+            rows.append((ph[0], ph[1], ph[2], rp[3]))
+            xl.copy_(zl + 1e-3)
+        m = np.median(np.array(rows[1:]), axis=0)
+        out["bylayer"] = {"n_elems": nl, "n_blocks": int(boff.size - 1), "longest_block": int(np.diff(boff.astype(np.int64)).max()),
+                          "scores_ms": float(m[0]), "scores_gbs": 2 * nl * ELEM / m[0] / 1e6,
+                          "select_ms": float(m[1]), "pack_ms": float(m[2]), "pack_gbs": 3 * pe * ELEM / m[2] / 1e6,
+                          "recover_ms": float(m[3]), "recover_gbs": 3 * le * ELEM / m[3] / 1e6, "lost_elems": le}
+        cl.close()
+    return out
 
 
 def run_e2e(api, ck, x0, z_lib, z0, r_sweep, lost_shards, lost_elems, n, nb, world, flush):
@@ -511,6 +623,8 @@ def main():
                     help="elements of the CNN-scale parameter vector (default 2**30)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the measurements beside the headline step (baseline selectors, drain, by-layer layout)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -131,7 +131,7 @@ template <typename P> int dev_alloc(scar_ctx *c, P **p, size_t bytes) {
 // Validates the caller's layout and fills the host-side fields of Geom
 // (boff is set later, once the offsets are on the device).
 int resolve_layout(const scar_layout *L, Geom &g) {
-    if (L->n_shards < 1) return SCAR_ERR_LAYOUT;
+    if (L->n_shards < 1 || L->n_elems >= (1ull << 48)) return SCAR_ERR_LAYOUT;
     g = Geom{};
     g.n_elems = L->n_elems;
     g.n_shards = L->n_shards;

@@ -127,6 +127,28 @@ template <typename W> __device__ __forceinline__ W cta_excl_scan(W v, W *sh /*kT
     return before + inc - v;
 }
 
+// Sums N values per thread over the CTA with one pair of barriers (the selection kernel is a chain of
+// short dependent phases, so barriers are what it pays for).  sh holds N * kThreads / 32 words.
+template <int N>
+__device__ __forceinline__ void cta_sum_n(unsigned long long (&v)[N], unsigned long long *sh) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+    for (int i = 0; i < N; ++i) v[i] = group_sum<32, unsigned long long>(v[i]);
+    __syncthreads();
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) sh[w * N + i] = v[i];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        unsigned long long t = 0;
+#pragma unroll
+        for (int j = 0; j < kThreads / 32; ++j) t += sh[j * N + i];
+        v[i] = t;
+    }
+}
+
 // Grid-wide barrier number `phase` (1, 2, ...) of a cooperative launch: every
 // CTA of the grid must call it the same number of times.  Returns false when
 // the wait was abandoned (it cannot happen while all CTAs are resident, which a
@@ -161,17 +183,19 @@ __device__ __forceinline__ bool grid_barrier(SelState *st, unsigned phase) {
 // Resolves one digit: scanning bins from the highest down, finds the bin d with
 //   count(bins > d) < remaining <= count(bins >= d)
 // and returns it; remaining becomes the rank wanted inside bin d.
-__device__ __forceinline__ unsigned resolve_digit(const unsigned *hist, int width, unsigned long long &remaining,
-                                                  unsigned long long *sh_scan, unsigned long long *sh_out) {
-    const int nb = 1 << width;
-    const int per = nb / kThreads;  // 8 or 4
-    unsigned local[kHistBins / kThreads];
+template <int WIDTH>
+__device__ __forceinline__ unsigned resolve_digit_w(const unsigned *hist, unsigned long long &remaining,
+                                                    unsigned long long *sh_scan, unsigned long long *sh_out) {
+    constexpr int nb = 1 << WIDTH;
+    constexpr int per = nb / kThreads;  // 8 or 4: a compile-time count, so all loads are in flight together
+    unsigned local[per];
     unsigned long long sum = 0;
-    for (int i = 0; i < per; ++i) {
-        local[i] = __ldcg(hist + (nb - 1 - (threadIdx.x * per + i)));
-        sum += local[i];
-    }
+#pragma unroll
+    for (int i = 0; i < per; ++i) local[i] = __ldcg(hist + (nb - 1 - (threadIdx.x * per + i)));
+#pragma unroll
+    for (int i = 0; i < per; ++i) sum += local[i];
     unsigned long long cum = cta_excl_scan<unsigned long long>(sum, sh_scan, nullptr);
+#pragma unroll
     for (int i = 0; i < per; ++i) {
         unsigned long long h = local[i];
         if (cum < remaining && remaining <= cum + h) {
@@ -185,6 +209,12 @@ __device__ __forceinline__ unsigned resolve_digit(const unsigned *hist, int widt
     unsigned d = (unsigned)sh_out[0];
     __syncthreads();
     return d;
+}
+
+__device__ __forceinline__ unsigned resolve_digit(const unsigned *hist, int width, unsigned long long &remaining,
+                                                  unsigned long long *sh_scan, unsigned long long *sh_out) {
+    return width == 11 ? resolve_digit_w<11>(hist, remaining, sh_scan, sh_out)
+                       : resolve_digit_w<10>(hist, remaining, sh_scan, sh_out);
 }
 
 // Flags of the kPerThread consecutive blocks a thread owns in tile t.
@@ -221,7 +251,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
     __shared__ unsigned sh_hist[kHistBins];
     __shared__ u64 sh_scan[kThreads / 32 + 1];
     __shared__ u64 sh_out[2];
-    __shared__ u64 sh_red[kThreads / 32];
+    __shared__ u64 sh_red[6 * kThreads / 32];
     __shared__ long long sh_boundary;
     __shared__ u64 sh_boundary_take;
     __shared__ bool sh_last;
@@ -287,11 +317,9 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
             c_eq += __popc(eq_bits);
             c_nf += __popc(nf_bits);
         }
-        c_gt = cta_sum<u64>(c_gt, sh_red);
-        c_eq = cta_sum<u64>(c_eq, sh_red);
-        c_nf = cta_sum<u64>(c_nf, sh_red);
-        lgt = cta_sum<u64>(lgt, sh_red);
-        leq = cta_sum<u64>(leq, sh_red);
+        u64 five[5] = {c_gt, c_eq, c_nf, lgt, leq};
+        cta_sum_n<5>(five, sh_red);
+        c_gt = five[0], c_eq = five[1], c_nf = five[2], lgt = five[3], leq = five[4];
         if (threadIdx.x == 0) {
             ca.gt[blockIdx.x] = (unsigned)c_gt;
             ca.eq[blockIdx.x] = (unsigned)c_eq;
@@ -335,14 +363,11 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
                 }
             }
         }
-        my_eq_before = cta_sum<u64>(a_eq, sh_red);
-        my_sel_base = cta_sum<u64>(a_n, sh_red);
-        my_len_base = cta_sum<u64>(a_l, sh_red);
-        total_n = cta_sum<u64>(t_n, sh_red);
-        total_l = cta_sum<u64>(t_l, sh_red);
-        total_nf = cta_sum<u64>(t_nf, sh_red);
-        __syncthreads();
-        cb = sh_boundary;
+        u64 six[6] = {a_eq, a_n, a_l, t_n, t_l, t_nf};
+        cta_sum_n<6>(six, sh_red);
+        my_eq_before = six[0], my_sel_base = six[1], my_len_base = six[2];
+        total_n = six[3], total_l = six[4], total_nf = six[5];
+        cb = sh_boundary;  // written before the barriers inside cta_sum_n
     }
 
     // ---- boundary CTA: summed length of the tau-blocks it takes (lowest ids first)
@@ -405,8 +430,14 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
                     lsum += len;
                 }
             }
-            u64 pos = pos_base + cta_excl_scan<u64>(__popc(take_bits), sh_scan, &tot_n);
-            u64 off = off_base + cta_excl_scan<u64>(lsum, sh_scan, &tot_l);
+            // one scan for both outputs: block counts in the top 16 bits (at most 2048 per tile), summed
+            // lengths below (a buffer has fewer than 2^48 elements: init rejects more)
+            u64 tot_both;
+            const u64 both = cta_excl_scan<u64>(((u64)__popc(take_bits) << 48) | lsum, sh_scan, &tot_both);
+            u64 pos = pos_base + (both >> 48);
+            u64 off = off_base + (both & ((1ull << 48) - 1));
+            tot_n = tot_both >> 48;
+            tot_l = tot_both & ((1ull << 48) - 1);
 #pragma unroll
             for (int j = 0; j < kPerThread; ++j)
                 if (take_bits >> j & 1u) {
