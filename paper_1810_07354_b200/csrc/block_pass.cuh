@@ -76,6 +76,13 @@ template <> struct Elem<int, kNormDefault> {
     static constexpr bool kFlush = false;
 };
 
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start while
+// the kernel before it is still running; it must call griddep_wait() before touching anything that kernel
+// writes.  griddep_launch() in the earlier kernel lets the later one be scheduled as soon as every CTA of the
+// earlier one has started.  Both are no-ops for launches without the attribute.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 template <typename V> __device__ __forceinline__ V ld_stream(const V *p) { return __ldcs(p); }
 template <typename V> __device__ __forceinline__ void st_stream(V *p, const V &v) { __stcs(p, v); }
 
@@ -235,6 +242,7 @@ __global__ void __launch_bounds__(kThreads)
 k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S, const float *__restrict__ weight,
                  typename Elem<T, NORM>::score_t *__restrict__ part) {
     using E = Elem<T, NORM>;
+    griddep_launch();  // the reduction that follows may be scheduled early; it waits for this grid before reading
     const int lane = threadIdx.x & (G - 1);
     if (G < 32 && S.mode == 2) {
         // Per-block mask with several blocks per warp: a warp takes 32 consecutive
@@ -312,6 +320,7 @@ k_reduce_partials(const typename Elem<T>::score_t *__restrict__ part, Geom g, Lo
     __shared__ double shd[kThreads / 32];
     __shared__ unsigned long long shu[kThreads / 32];
     __shared__ bool is_last;
+    griddep_wait();
     const uint64_t base = (uint64_t)blockIdx.x * kReduceTile;
     double fs = 0.0;
     unsigned long long is = 0, nb = 0, ne = 0;

@@ -52,6 +52,7 @@ k_pack_update(const uint32_t *__restrict__ x, uint32_t *__restrict__ z, uint32_t
     const int lane = threadIdx.x & (G - 1);
     const uint64_t j = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
     if (j >= k) return;
+    griddep_wait();  // the selection that wrote sel / poff may still be running
     uint64_t beg, len;
     g.range(sel[j], beg, len);
     const uint64_t dst = poff[j];

@@ -204,6 +204,22 @@ unsigned grid_for_groups(uint64_t n_groups, int G) {
     return (unsigned)((n_groups + per_cta - 1) / per_cta);
 }
 
+// Launch that may overlap the tail of the kernel before it on the stream (the kernel calls griddep_wait()
+// before it reads that kernel's output).  Off while per-phase timing is on: phases would blur.
+template <typename... KArgs, typename... Args>
+void launch_after(scar_ctx *c, void (*kern)(KArgs...), unsigned grid, Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = c->profile ? 0 : 1;
+    cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 void record(scar_ctx *c, int i) {
     if (c->profile) cudaEventRecord(c->ev[i], c->stream);
 }
@@ -317,9 +333,9 @@ void launch_pack(scar_ctx *c, uint64_t k) {
     dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
         constexpr int G = decltype(gl)::value;
         constexpr bool VEC = decltype(vec)::value;
-        k_pack_update<G, VEC><<<grid_for_groups(k, G), kThreads, 0, c->stream>>>(
-            static_cast<const uint32_t *>(c->x), static_cast<uint32_t *>(c->z), static_cast<uint32_t *>(c->cur.payload),
-            c->g, c->cur.sel, c->cur.poff, k);
+        launch_after(c, k_pack_update<G, VEC>, grid_for_groups(k, G), static_cast<const uint32_t *>(c->x),
+                     static_cast<uint32_t *>(c->z), static_cast<uint32_t *>(c->cur.payload), c->g, c->cur.sel,
+                     c->cur.poff, (unsigned long long)k);
     });
     ++c->launches;
 }
@@ -365,9 +381,8 @@ template <typename T, int NORM> void launch_recover_as(scar_ctx *c, const LostSe
     record(c, 4);
     uint64_t tiles = (S.n_work + kReduceTile - 1) / kReduceTile;
     if (tiles == 0) tiles = 1;
-    k_reduce_partials<T><<<(unsigned)tiles, kThreads, 0, c->stream>>>(
-        static_cast<const Sc *>(c->part), c->g, S, c->rt_sum, c->rt_l1, c->rt_blocks, c->rt_elems,
-        &c->st->ticket_reduce, c->d_norm, NORM == kNormDefault);
+    launch_after(c, k_reduce_partials<T>, (unsigned)tiles, static_cast<const Sc *>(c->part), c->g, S, c->rt_sum,
+                 c->rt_l1, c->rt_blocks, c->rt_elems, &c->st->ticket_reduce, c->d_norm, NORM == kNormDefault);
     ++c->launches;
     record(c, 5);
 }

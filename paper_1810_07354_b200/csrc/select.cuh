@@ -256,6 +256,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
     __shared__ u64 sh_boundary_take;
     __shared__ bool sh_last;
 
+    griddep_launch();  // the pack kernel may be scheduled while this one runs; it waits before reading sel / poff
     const u64 B = g.n_blocks;
     const unsigned t_lo = blockIdx.x * tiles_per_cta;
     const unsigned t_hi = t_lo + tiles_per_cta < n_tiles ? t_lo + tiles_per_cta : n_tiles;
