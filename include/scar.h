@@ -308,6 +308,18 @@ double scar_discounted_perturbation(const double *norms, const uint64_t *iters, 
 double scar_iteration_cost_bound(double delta_T, double dist0, double c);
 double scar_irreducible_error(double delta_max, double c);
 
+/* Self-test hook for the bounded device-side wait.  The selection kernel's
+ * CTAs meet at grid barriers whose wait gives up after a fixed number of tries
+ * instead of hanging.  This call mis-sets the barrier's arrival counter (nothing
+ * else), so that the first barrier of the NEXT prioritized or random save can
+ * never complete: that save takes about a second (the length of the bounded
+ * wait), selects and copies nothing, leaves z untouched, and returns
+ * SCAR_ERR_TIMEOUT from the call that reads its result (the save itself with a
+ * non-NULL out, or scar_ckpt_last_info).  The kernel puts the barrier state back
+ * on its way out, so the save after that one works normally.  Enqueue only.
+ * SCAR_ERR_STATE on an empty buffer. */
+int scar_ckpt_selftest_arm_timeout(scar_ctx *ctx);
+
 /* Waits for the stream, frees everything the context owns (never x). */
 int scar_ckpt_destroy(scar_ctx *ctx);
 

@@ -92,6 +92,7 @@ _SIGS = {
     "scar_discounted_perturbation": (_dbl, [_vp, _vp, _u64, _dbl]),
     "scar_iteration_cost_bound": (_dbl, [_dbl, _dbl, _dbl]),
     "scar_irreducible_error": (_dbl, [_dbl, _dbl]),
+    "scar_ckpt_selftest_arm_timeout": (_int, [_vp]),
     "scar_ckpt_destroy": (_int, [_vp]),
     "scar_strerror": (C.c_char_p, [_int]),
 }
@@ -345,6 +346,10 @@ def scar_iteration_cost_bound(delta_T: float, dist0: float, c: float) -> float:
 
 def scar_irreducible_error(delta_max: float, c: float) -> float:
     return float(load_library().scar_irreducible_error(delta_max, c))
+
+
+def scar_ckpt_selftest_arm_timeout(ctx: int) -> None:
+    _check(load_library().scar_ckpt_selftest_arm_timeout(ctx), "scar_ckpt_selftest_arm_timeout")
 
 
 def scar_ckpt_destroy(ctx: int) -> None:

@@ -48,11 +48,13 @@ __device__ __forceinline__ void copy_block_2dst(const U *__restrict__ src, U *__
 template <int G, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 k_pack_update(const uint32_t *__restrict__ x, uint32_t *__restrict__ z, uint32_t *__restrict__ payload, Geom g,
-              const uint32_t *__restrict__ sel, const unsigned long long *__restrict__ poff, unsigned long long k) {
+              const uint32_t *__restrict__ sel, const unsigned long long *__restrict__ poff, unsigned long long k,
+              const unsigned long long *selected) {
     const int lane = threadIdx.x & (G - 1);
     const uint64_t j = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
     if (j >= k) return;
     griddep_wait();  // the selection that wrote sel / poff may still be running
+    if (j >= *selected) return;  // fewer blocks than asked for: only when the selection gave up (then 0)
     uint64_t beg, len;
     g.range(sel[j], beg, len);
     const uint64_t dst = poff[j];

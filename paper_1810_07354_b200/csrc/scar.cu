@@ -335,7 +335,7 @@ void launch_pack(scar_ctx *c, uint64_t k) {
         constexpr bool VEC = decltype(vec)::value;
         launch_after(c, k_pack_update<G, VEC>, grid_for_groups(k, G), static_cast<const uint32_t *>(c->x),
                      static_cast<uint32_t *>(c->z), static_cast<uint32_t *>(c->cur.payload), c->g, c->cur.sel,
-                     c->cur.poff, (unsigned long long)k);
+                     c->cur.poff, (unsigned long long)k, &c->cur.info->k);
     });
     ++c->launches;
 }
@@ -930,6 +930,18 @@ int scar_ckpt_set_norm(scar_ctx *c, scar_norm norm, const float *h_block_weights
         c->d_weight = nullptr;
     }
     c->norm = norm;
+    return SCAR_OK;
+}
+
+int scar_ckpt_selftest_arm_timeout(scar_ctx *c) {
+    if (!c) return SCAR_ERR_INVALID_ARG;
+    if (c->g.n_blocks == 0) return SCAR_ERR_STATE;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    // An arrival counter that starts just below zero wraps to a small number after the first arrivals and
+    // then never reaches the first barrier's target, so every CTA's wait runs out.
+    static const unsigned biased = 0u - 1u;
+    CU_TRY(cudaMemcpyAsync(&c->st->barrier, &biased, sizeof(unsigned), cudaMemcpyHostToDevice, c->stream));
     return SCAR_OK;
 }
 

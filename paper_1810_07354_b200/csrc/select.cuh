@@ -473,6 +473,10 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
     if (threadIdx.x == 0) {
         const unsigned err = *reinterpret_cast<volatile unsigned *>(&st->error);
         info->error = err;
+        if (err) {  // a barrier gave up: nothing was selected, and the pack kernel must copy nothing
+            info->k = 0;
+            info->payload_elems = 0;
+        }
         st->key_or = 0;  // forget which uint64 key bits were seen
         st->barrier = 0;
         st->departed = 0;

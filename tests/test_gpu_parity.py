@@ -457,3 +457,37 @@ def test_empty_buffer():
     n = ck.recover_partial(np.ones(4, np.uint8))
     assert (n.l2, int(n.lost_blocks)) == (0.0, 0)
     ck.close()
+
+
+# ------------------------------------------------------------------ the bounded wait
+
+
+@pytest.mark.parametrize("kind", ["f32", "i32"])
+def test_a_barrier_that_cannot_complete_times_out_and_the_context_survives(kind):
+    """The selection's grid barrier gives up after a bounded number of tries: the save reports a timeout, has
+    copied nothing, and the next save is exact again.  The wait is made to run out by mis-setting the arrival
+    counter (a flag that nothing sets), never by a fault."""
+    w = make_workload("tiny", n_elems=1 << 20) if kind == "f32" else make_workload("lda", vocab=20_000, topics=100)
+    boff = block_offsets(w.geom)
+    xd = parity.to_dev(w.x)
+    ck = parity.make_ctx(xd, w.z, geom=w.geom)
+    k = w.n_blocks // 4
+    api.scar_ckpt_selftest_arm_timeout(ck.ctx)
+    with pytest.raises(api.ScarError) as e:
+        ck.priority_save_k(k)
+    assert e.value.code == -6 and "wait" in str(e.value)
+    assert parity.same_bits(ck.views()["z"].cpu().numpy(), w.z), "a save that timed out must not touch z"
+    assert xd.cpu().numpy().tobytes() == w.x.tobytes()
+    ora = oracle.priority_save(w.x, w.z, boff, k=k)
+    parity.check_save(ck, ck.priority_save_k(k), w.x, w.z, boff, ora)
+    # armed again, read through last_info after an enqueue-only save; then a random save goes through
+    api.scar_ckpt_selftest_arm_timeout(ck.ctx)
+    ck.priority_save_k(k, sync=False)
+    with pytest.raises(api.ScarError) as e:
+        api.scar_ckpt_last_info(ck.ctx, True, False)
+    assert e.value.code == -6
+    pri = rng(3).integers(0, 2**32, size=w.n_blocks, dtype=np.uint64).astype(np.uint32)
+    info = ck.save_random(5, parity.to_dev(pri.view(np.int32)))
+    assert int(info.k) == 5
+    np.testing.assert_array_equal(parity.fetch_save(ck, info)["sel"], oracle.select_random(pri, 5))
+    ck.close()
