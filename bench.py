@@ -406,7 +406,7 @@ def run_gpu(args):
         ms = float(np.median(t[("save", r)]))
         by = save_bytes(n, payload_elems[r])
         ph = np.median(np.array(phase[r]), axis=0)
-        per_r[str(r)] = {"save_ms": ms, "scanned_gbs": scanned / ms / 1e6, "algorithmic_gbs": by / ms / 1e6,
+        per_r[str(r)] = {"save_ms": ms, "save_ms_min": float(np.min(t[("save", r)])), "scanned_gbs": scanned / ms / 1e6, "algorithmic_gbs": by / ms / 1e6,
                          "frac_of_measured_peak": by / ms / 1e6 / peak, "frac_of_8tbs": by / ms / 1e6 / 8000.0,
                          "blocks_per_s": nb / (ms * 1e-3), "payload_elems": payload_elems[r],
                          "phase_ms": {"scores": float(ph[0]), "select": float(ph[1]), "pack": float(ph[2])}}
