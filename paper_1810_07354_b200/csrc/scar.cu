@@ -282,6 +282,19 @@ void launch_scores(scar_ctx *c) {
     else launch_scores_as<float, kNormDefault>(c);
 }
 
+// a1 + a3 fused for k == B
+template <typename T, int NORM> void launch_full_save(scar_ctx *c) {
+    using S = typename Elem<T, NORM>::score_t;
+    dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
+        constexpr int G = decltype(gl)::value;
+        constexpr bool VEC = decltype(vec)::value;
+        k_full_save<T, NORM, G, VEC><<<grid_for_groups(c->g.n_blocks, G), kThreads, 0, c->stream>>>(
+            static_cast<const T *>(c->x), static_cast<T *>(c->z), static_cast<T *>(c->cur.payload), c->g, c->d_weight,
+            static_cast<S *>(c->score), c->cur.sel, c->cur.poff, c->cur.info);
+    });
+    ++c->launches;
+}
+
 // a2: one cooperative launch (all CTAs resident, so its grid-wide barriers cannot deadlock)
 template <typename S> int launch_select(scar_ctx *c, const S *score, uint64_t k) {
     unsigned long long kk = k;
@@ -460,6 +473,20 @@ int enqueue_save(scar_ctx *c, uint64_t k) {
     if (c->g.n_blocks == 0) {
         CU_TRY(cudaMemsetAsync(c->cur.info, 0, sizeof(SaveInfoDev), c->stream));
         CU_TRY(cudaMemsetAsync(c->cur.poff, 0, sizeof(unsigned long long), c->stream));
+        c->have_save = true;
+        return SCAR_OK;
+    }
+    if (k == c->g.n_blocks && !c->seg_mode) {
+        // Full checkpoint: nothing to choose, so one fused pass scores, packs and refreshes z.
+        CU_TRY(cudaMemsetAsync(c->cur.info, 0, sizeof(SaveInfoDev), c->stream));
+        if (c->dt == SCAR_I32) launch_full_save<int, kNormDefault>(c);
+        else if (c->norm == SCAR_NORM_L1) launch_full_save<float, kNormL1>(c);
+        else launch_full_save<float, kNormDefault>(c);
+        record(c, 1);
+        record(c, 2);
+        record(c, 3);
+        c->ran_select = c->ran_pack = true;
+        CU_TRY(cudaGetLastError());
         c->have_save = true;
         return SCAR_OK;
     }

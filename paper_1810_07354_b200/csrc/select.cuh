@@ -484,6 +484,93 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
     }
 }
 
+// ---- the traditional full checkpoint (k == B) -----------------------------------
+//
+// When every block is saved the selection is known beforehand (all ids, in
+// order, each block's payload offset equal to its own offset), so scoring and
+// packing fuse into one pass: x and z are read once for the distance, and x is
+// written to the payload and over z from the registers it already sits in.
+// That moves 4 N elements instead of the 5 N of score pass + pack pass.
+// Same traversal and accumulation order as block_distance, so the scores are
+// bit-identical to a partial save's.
+template <typename T, int NORM, int G, bool VEC>
+__device__ __forceinline__ typename Elem<T, NORM>::wide_t block_distance_save(const T *__restrict__ x, T *__restrict__ z,
+                                                                              T *__restrict__ payload, uint64_t beg,
+                                                                              uint64_t len, int lane) {
+    using E = Elem<T, NORM>;
+    using U = typename std::conditional<VEC, typename E::vec_t, T>::type;
+    using acc_t = typename E::acc_t;
+    using wide_t = typename E::wide_t;
+    constexpr unsigned kFlushMask = VEC ? 63u : 255u;
+    const U *xs = reinterpret_cast<const U *>(x + beg);
+    U *zs = reinterpret_cast<U *>(z + beg);
+    U *ps = reinterpret_cast<U *>(payload + beg);
+    const uint64_t n = VEC ? (len >> 2) : len;
+    constexpr uint64_t step = 4 * (uint64_t)G;
+    acc_t a[4] = {0, 0, 0, 0};
+    wide_t total = 0;
+    U xc[4], zc[4], xn[4], zn[4];
+    uint64_t u = lane;
+    unsigned it = 0;
+    bool have = u < n;
+    if (have) load_batch<U, G>(xs, zs, u, n, xc, zc);
+    while (have) {  // loads of the next batch are issued before the stores of this one (see block_distance)
+        const uint64_t un = u + step;
+        const bool more = un < n;
+        if (more) load_batch<U, G>(xs, zs, un, n, xn, zn);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            E::addu(a[j], xc[j], zc[j]);
+            const uint64_t i = u + (uint64_t)j * G;
+            if (i < n) {
+                st_stream(ps + i, xc[j]);
+                st_stream(zs + i, xc[j]);
+            }
+        }
+        if (E::kFlush && (++it & kFlushMask) == 0) {
+            total += ((wide_t)a[0] + (wide_t)a[1]) + ((wide_t)a[2] + (wide_t)a[3]);
+            a[0] = a[1] = a[2] = a[3] = 0;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            xc[j] = xn[j];
+            zc[j] = zn[j];
+        }
+        u = un;
+        have = more;
+    }
+    total += ((wide_t)a[0] + (wide_t)a[1]) + ((wide_t)a[2] + (wide_t)a[3]);
+    return group_sum<G, wide_t>(total);
+}
+
+// info must have been cleared before the launch (the non-finite count is added up with atomics).
+template <typename T, int NORM, int G, bool VEC>
+__global__ void __launch_bounds__(kThreads)
+k_full_save(const T *__restrict__ x, T *__restrict__ z, T *__restrict__ payload, Geom g, const float *__restrict__ weight,
+            typename Elem<T, NORM>::score_t *__restrict__ score, uint32_t *__restrict__ sel,
+            unsigned long long *__restrict__ poff, SaveInfoDev *info) {
+    using E = Elem<T, NORM>;
+    using SK = ScoreKey<typename E::score_t>;
+    const int lane = threadIdx.x & (G - 1);
+    const uint64_t grp = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
+    const bool valid = grp < g.n_blocks;
+    uint64_t beg = 0, len = 0;
+    if (valid) g.range((uint32_t)grp, beg, len);
+    typename E::wide_t s = block_distance_save<T, NORM, G, VEC>(x, z, payload, beg, len, lane);
+    if (valid && lane == 0) {
+        const typename E::score_t sc = weighted<E>(s, weight, grp);
+        score[grp] = sc;
+        sel[grp] = (uint32_t)grp;
+        poff[grp] = beg;
+        if (SK::nonfinite(SK::key(sc))) atomicAdd(&info->nonfinite_blocks, 1ull);
+        if (grp == g.n_blocks - 1) {
+            poff[g.n_blocks] = g.n_elems;
+            info->k = g.n_blocks;
+            info->payload_elems = g.n_elems;
+        }
+    }
+}
+
 // ---- baseline strategies of Section 5.4 -------------------------------------
 //
 // `round`: the k blocks that follow a cursor, wrapping at the end of the buffer.
