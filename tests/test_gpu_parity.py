@@ -491,3 +491,52 @@ def test_a_barrier_that_cannot_complete_times_out_and_the_context_survives(kind)
     assert int(info.k) == 5
     np.testing.assert_array_equal(parity.fetch_save(ck, info)["sel"], oracle.select_random(pri, 5))
     ck.close()
+
+
+# ------------------------------------------------------------------ several contexts at once
+
+
+def test_two_contexts_on_two_streams_run_side_by_side():
+    """Each context has its own stream and its own work arrays; saves and recoveries enqueued on both without
+    waiting in between (the selection kernels are cooperative launches that may have to take turns) give the same
+    bytes as when each runs alone."""
+    wa = make_workload("tiny", n_elems=1 << 22, seed=11)
+    wb = make_workload("lda", vocab=30_000, topics=200, seed=12)
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    xa, xb = parity.to_dev(wa.x), parity.to_dev(wb.x)
+    za, zb = parity.to_dev(wa.z), parity.to_dev(wb.z)
+    torch.cuda.synchronize()
+    ca = api.ScarCheckpoint(xa, n_shards=8, block_elems=wa.geom.block_elems, stream=sa)
+    cb = api.ScarCheckpoint(xb, n_shards=8, row_elems=wb.geom.row_elems, block_elems=wb.geom.block_elems, stream=sb)
+    boa, bob = block_offsets(wa.geom), block_offsets(wb.geom)
+    ka, kb = wa.n_blocks // 4, wb.n_blocks // 5
+    ora_a = oracle.priority_save(wa.x, wa.z, boa, k=ka)
+    ora_b = oracle.priority_save(wb.x, wb.z, bob, k=kb)
+    for rep in range(5):
+        ca.load(za)
+        cb.load(zb)
+        for _ in range(3):  # back-to-back saves on both streams, nothing waits
+            ca.priority_save_k(ka, sync=False)
+            cb.priority_save_k(kb, sync=False)
+        ca.load(za)
+        cb.load(zb)
+        ca.priority_save_k(ka, sync=False)
+        cb.priority_save_k(kb, sync=False)
+        ia, _ = api.scar_ckpt_last_info(ca.ctx, True, False)
+        ib, _ = api.scar_ckpt_last_info(cb.ctx, True, False)
+        parity.check_save(ca, ia, wa.x, wa.z, boa, ora_a)
+        parity.check_save(cb, ib, wb.x, wb.z, bob, ora_b)
+    ca.load(za)
+    cb.load(zb)
+    ca.recover_partial(wa.lost_shards, sync=False)
+    cb.recover_partial(wb.lost_shards, sync=False)
+    _, na = api.scar_ckpt_last_info(ca.ctx, False, True)
+    _, nb_ = api.scar_ckpt_last_info(cb.ctx, False, True)
+    want_a, xa_after = oracle.recover_partial(wa.x, wa.z, boa, oracle.expand_shards(wa.n_blocks, wa.lost_shards))
+    want_b, xb_after = oracle.recover_partial(wb.x, wb.z, bob, oracle.expand_shards(wb.n_blocks, wb.lost_shards))
+    parity.check_norm(na, want_a, True)
+    parity.check_norm(nb_, want_b, False)
+    torch.cuda.synchronize()
+    assert xa.cpu().numpy().tobytes() == xa_after.tobytes() and xb.cpu().numpy().tobytes() == xb_after.tobytes()
+    ca.close()
+    cb.close()
