@@ -24,6 +24,9 @@
  *   - All GPU work of a context runs on the CUDA stream given at init, in call
  *     order.  A call whose result pointer `out` is NULL only enqueues; with a
  *     non-NULL `out` it also waits for the stream and fills `out`.
+ *     Enqueue-only calls use no host synchronisation and can be recorded by
+ *     CUDA stream capture on the context's stream (saves, recoveries with
+ *     shard masks or device block masks, norms, scar_ckpt_load).
  *   - One context serves one caller at a time (no internal locking).
  *   - There is no CPU fallback: without a usable CUDA device init fails.
  */

@@ -540,3 +540,34 @@ def test_two_contexts_on_two_streams_run_side_by_side():
     assert xa.cpu().numpy().tobytes() == xa_after.tobytes() and xb.cpu().numpy().tobytes() == xb_after.tobytes()
     ca.close()
     cb.close()
+
+
+def test_enqueue_only_calls_can_be_captured_in_a_cuda_graph():
+    """Calls with a NULL result pointer only enqueue, so a reload + save + recovery sequence can be captured once
+    and replayed; every replay gives the oracle's bytes."""
+    w = make_workload("tiny", n_elems=1 << 20)
+    boff = block_offsets(w.geom)
+    s = torch.cuda.Stream()
+    x, z0 = parity.to_dev(w.x), parity.to_dev(w.z)
+    x0 = x.clone()
+    torch.cuda.synchronize()
+    ck = api.ScarCheckpoint(x, n_shards=8, block_elems=w.geom.block_elems, stream=s)
+    k = w.n_blocks // 4
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        ck.load(z0)
+        ck.priority_save_k(k, sync=False)
+        ck.recover_partial(w.lost_shards, sync=False)
+    ora = oracle.priority_save(w.x, w.z, boff, k=k)
+    lost = oracle.expand_shards(w.n_blocks, w.lost_shards)
+    for _ in range(3):
+        x.copy_(x0)
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        info, nrm = api.scar_ckpt_last_info(ck.ctx)
+        got = parity.check_save(ck, info, w.x, w.z, boff, ora)
+        want, x_after = oracle.recover_partial(w.x, got["z"], boff, lost)
+        parity.check_norm(nrm, want, True)
+        assert x.cpu().numpy().tobytes() == x_after.tobytes()
+    ck.close()
