@@ -151,6 +151,17 @@ def check_save(ck: api.ScarCheckpoint, info, x: np.ndarray, z_before: np.ndarray
     return got
 
 
+def next_checkpoint(z_before: np.ndarray, x: np.ndarray, boff: np.ndarray, got: dict, ora: "oracle.SaveResult"):
+    """The running checkpoint the oracle twin continues from after a checked save: the oracle's own when the ids
+    were the oracle's, else the oracle's update step applied to the ids the library chose inside the tolerance
+    band (already validated).  Never a buffer copied from the device."""
+    if got["exact"]:
+        return ora.z_after
+    z = z_before.copy()
+    oracle.update(z, x, boff, np.ascontiguousarray(got["sel"], dtype=np.uint32))
+    return z
+
+
 def check_norm(info, ora: "oracle.NormResult", is_float: bool):
     assert int(info.lost_blocks) == ora.lost_blocks
     assert int(info.lost_elems) == ora.lost_elems

@@ -120,7 +120,7 @@ def test_implicit_layout_with_huge_blocks_uses_the_same_path():
     got = parity.check_save(ck, ck.priority_save_k(5), x, z, boff, ora)
     assert got["scores"][5] == 0.0
     shards = np.array([1, 0, 1], dtype=np.uint8)
-    want, x_after = oracle.recover_partial(x, ora.z_after if got["exact"] else got["z"], boff, oracle.expand_shards(12, shards))
+    want, x_after = oracle.recover_partial(x, parity.next_checkpoint(z, x, boff, got, ora), boff, oracle.expand_shards(12, shards))
     parity.check_norm(ck.recover_partial(shards), want, True)
     assert xd.cpu().numpy().tobytes() == x_after.tobytes()
     ck.close()

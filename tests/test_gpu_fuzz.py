@@ -96,7 +96,7 @@ def test_random_case(seed):
         if which == "priority":
             ora = oracle_save(x, hz, boff, k, norm, w)
             got = parity.check_save(ck, ck.priority_save_k(k), x, hz, boff, ora, linear=linear)
-            hz = got["z"].copy()
+            hz = parity.next_checkpoint(hz, x, boff, got, ora)
         else:
             if which == "round":
                 sel, cursor = oracle.select_round(nb, k, cursor)

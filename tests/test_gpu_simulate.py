@@ -41,7 +41,7 @@ def test_simulation_in_lockstep_with_the_oracle(strategy):
             if strategy == "priority":
                 ora = oracle.priority_save(hx, hz, boff, k=sim.k)
                 got = parity.check_save(sim.ck, info, hx, hz, boff, ora)
-                hz = got["z"].copy()  # the validated ids decide what the checkpoint now holds
+                hz = parity.next_checkpoint(hz, hx, boff, got, ora)  # the validated ids decide what it holds
             else:
                 if strategy == "round":
                     sel, cursor = oracle.select_round(nb, sim.k, cursor)
