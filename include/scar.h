@@ -63,7 +63,8 @@ enum {
     SCAR_ERR_STATE = -5,       /* call not valid in the context's current state */
     SCAR_ERR_TIMEOUT = -6,     /* a bounded device-side wait (grid barrier of the selection) gave up;
                                   the save's outputs are invalid, the context stays usable */
-    SCAR_ERR_CAPACITY = -7     /* problem larger than a fixed-size internal buffer */
+    SCAR_ERR_CAPACITY = -7,    /* problem larger than a fixed-size internal buffer */
+    SCAR_ERR_IO = -8           /* a read or write of the stored checkpoint failed or came up short */
 };
 
 /* Block geometry of the flat buffer of n_elems elements.
@@ -259,6 +260,28 @@ int scar_ckpt_drain_enqueue(scar_ctx *ctx, uint64_t *ticket);
 int scar_ckpt_drain_done(scar_ctx *ctx, uint64_t ticket);
 int scar_ckpt_drain_wait(scar_ctx *ctx, uint64_t ticket, scar_drain_view *out);
 int scar_ckpt_drain_release(scar_ctx *ctx, uint64_t ticket);
+
+/* ---- The running checkpoint in persistent storage (Sections 4.2, 4.3) --------
+ * The paper keeps the running checkpoint in shared persistent storage and z is
+ * only the in-memory cache of it: step 4 of a checkpoint saves the selected
+ * parameters there, and a recovery re-loads parameters from it.  Here the
+ * stored checkpoint is a plain file of n_elems * 4 bytes in element order, given
+ * as an open POSIX file descriptor (the caller opens, syncs and closes it); after
+ * every store it holds exactly the bytes of z.
+ *   store_full     writes all of z (the initial checkpoint x^(0), or after
+ *                  scar_ckpt_load).  Waits for the stream.
+ *   store_drained  waits for the drain of `ticket` and writes each saved block
+ *                  from the pinned host mirror to its place in the file (one
+ *                  write per run of consecutive blocks).  The ticket stays
+ *                  valid; release it afterwards.  Host work only.
+ *   load_stored    z := the file (a restart that lost the in-memory cache, or a
+ *                  recovery from storage: follow it with scar_recover_partial).
+ *                  Waits for the stream.
+ * SCAR_ERR_IO on a failed or short read / write; the file or z may then be
+ * partly updated. */
+int scar_ckpt_store_full(scar_ctx *ctx, int fd);
+int scar_ckpt_store_drained(scar_ctx *ctx, uint64_t ticket, int fd);
+int scar_ckpt_load_stored(scar_ctx *ctx, int fd);
 
 /* Replaces the running checkpoint by n_elems elements read from the device
  * buffer d_z_src (e.g. a checkpoint read back from storage).  Enqueue only. */

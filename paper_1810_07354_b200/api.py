@@ -81,6 +81,9 @@ _SIGS = {
     "scar_ckpt_drain_done": (_int, [_vp, _u64]),
     "scar_ckpt_drain_wait": (_int, [_vp, _u64, C.POINTER(scar_drain_view)]),
     "scar_ckpt_drain_release": (_int, [_vp, _u64]),
+    "scar_ckpt_store_full": (_int, [_vp, _int]),
+    "scar_ckpt_store_drained": (_int, [_vp, _u64, _int]),
+    "scar_ckpt_load_stored": (_int, [_vp, _int]),
     "scar_ckpt_load": (_int, [_vp, _vp]),
     "scar_ckpt_last_info": (_int, [_vp, C.POINTER(scar_save_info), C.POINTER(scar_norm_info)]),
     "scar_ckpt_view": (_int, [_vp] + [C.POINTER(_vp)] * 5),
@@ -291,6 +294,18 @@ def scar_ckpt_drain_release(ctx: int, ticket: int) -> None:
     _check(load_library().scar_ckpt_drain_release(ctx, ticket), "scar_ckpt_drain_release")
 
 
+def scar_ckpt_store_full(ctx: int, fd: int) -> None:
+    _check(load_library().scar_ckpt_store_full(ctx, fd), "scar_ckpt_store_full")
+
+
+def scar_ckpt_store_drained(ctx: int, ticket: int, fd: int) -> None:
+    _check(load_library().scar_ckpt_store_drained(ctx, ticket, fd), "scar_ckpt_store_drained")
+
+
+def scar_ckpt_load_stored(ctx: int, fd: int) -> None:
+    _check(load_library().scar_ckpt_load_stored(ctx, fd), "scar_ckpt_load_stored")
+
+
 def scar_ckpt_load(ctx: int, d_z_src) -> None:
     _check(load_library().scar_ckpt_load(ctx, _addr(d_z_src)), "scar_ckpt_load")
 
@@ -457,6 +472,15 @@ class ScarCheckpoint:
 
     def drain_release(self, ticket: int):
         scar_ckpt_drain_release(self.ctx, ticket)
+
+    def store_full(self, fd: int):
+        scar_ckpt_store_full(self.ctx, fd)
+
+    def store_drained(self, ticket: int, fd: int):
+        scar_ckpt_store_drained(self.ctx, ticket, fd)
+
+    def load_stored(self, fd: int):
+        scar_ckpt_load_stored(self.ctx, fd)
 
     def load(self, d_z_src):
         scar_ckpt_load(self.ctx, d_z_src)

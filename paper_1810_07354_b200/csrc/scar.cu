@@ -2,6 +2,7 @@
 // the extern "C" entry points declared in include/scar.h.  Every step of the
 // checkpoint / recovery pass runs in the kernels of block_pass.cuh, select.cuh
 // and pack.cuh; there is no CPU path.
+#include <cerrno>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -9,6 +10,8 @@
 #include <new>
 #include <type_traits>
 #include <vector>
+
+#include <unistd.h>
 
 #include "scar.h"
 
@@ -91,6 +94,10 @@ struct scar_ctx {
     cudaStream_t drain_stream = nullptr;
     uint64_t drain_cap_k = 0, drain_cap_elems = 0, next_ticket = 0;
     uint64_t max_block_len = 0;
+
+    // persistent copy of the running checkpoint (scar_ckpt_store_* / scar_ckpt_load_stored)
+    std::vector<uint64_t> h_boff;  // host copy of explicit block offsets (empty for implicit layouts)
+    char *io_stage = nullptr;      // pinned staging buffer for whole-checkpoint transfers
 
     std::vector<void *> owned;  // device allocations to free
     std::vector<void *> owned_host;  // pinned host allocations to free
@@ -654,6 +661,7 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     c->x = d_x;
     c->group_lanes = pick_group_lanes(g);
     if (layout->block_offsets) {
+        c->h_boff.assign(layout->block_offsets, layout->block_offsets + g.n_blocks + 1);
         for (uint64_t b = 0; b < g.n_blocks; ++b) {
             const uint64_t len = layout->block_offsets[b + 1] - layout->block_offsets[b];
             if (len > c->max_block_len) c->max_block_len = len;
@@ -1093,6 +1101,123 @@ int scar_ckpt_drain_release(scar_ctx *c, uint64_t ticket) {
     return SCAR_OK;
 }
 
+// ---- the running checkpoint in persistent storage (Sections 4.2, 4.3) ---------------------------
+
+namespace {
+
+constexpr size_t kIoStageBytes = 64u << 20;
+
+void host_range(const scar_ctx *c, uint64_t b, uint64_t &beg, uint64_t &len) {
+    if (!c->h_boff.empty()) {
+        beg = c->h_boff[b];
+        len = c->h_boff[b + 1] - beg;
+        return;
+    }
+    const uint64_t row = b / c->g.blocks_per_row, j = b % c->g.blocks_per_row, o = j * c->g.block_elems;
+    beg = row * c->g.row_len + o;
+    len = c->g.row_len - o < c->g.block_elems ? c->g.row_len - o : c->g.block_elems;
+}
+
+int write_all(int fd, const char *p, size_t n, uint64_t off) {
+    while (n) {
+        const ssize_t w = pwrite(fd, p, n, (off_t)off);
+        if (w < 0) {
+            if (errno == EINTR) continue;
+            return SCAR_ERR_IO;
+        }
+        if (w == 0) return SCAR_ERR_IO;
+        p += w;
+        n -= (size_t)w;
+        off += (uint64_t)w;
+    }
+    return SCAR_OK;
+}
+
+int read_all(int fd, char *p, size_t n, uint64_t off) {
+    while (n) {
+        const ssize_t r = pread(fd, p, n, (off_t)off);
+        if (r < 0) {
+            if (errno == EINTR) continue;
+            return SCAR_ERR_IO;
+        }
+        if (r == 0) return SCAR_ERR_IO;  // the file is shorter than the checkpoint
+        p += r;
+        n -= (size_t)r;
+        off += (uint64_t)r;
+    }
+    return SCAR_OK;
+}
+
+int ensure_stage(scar_ctx *c) {
+    if (c->io_stage) return SCAR_OK;
+    void *q = nullptr;
+    if (cudaMallocHost(&q, kIoStageBytes) != cudaSuccess) {
+        cudaGetLastError();
+        return SCAR_ERR_ALLOC;
+    }
+    c->owned_host.push_back(q);
+    c->io_stage = static_cast<char *>(q);
+    return SCAR_OK;
+}
+
+}  // namespace
+
+int scar_ckpt_store_full(scar_ctx *c, int fd) {
+    if (!c || fd < 0) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc == SCAR_OK) rc = ensure_stage(c);
+    if (rc != SCAR_OK) return rc;
+    const uint64_t bytes = c->g.n_elems * 4;
+    const char *z = static_cast<const char *>(c->z);
+    for (uint64_t off = 0; off < bytes; off += kIoStageBytes) {
+        const size_t n = (size_t)(bytes - off < kIoStageBytes ? bytes - off : kIoStageBytes);
+        CU_TRY(cudaMemcpyAsync(c->io_stage, z + off, n, cudaMemcpyDeviceToHost, c->stream));
+        CU_TRY(cudaStreamSynchronize(c->stream));
+        if ((rc = write_all(fd, c->io_stage, n, off)) != SCAR_OK) return rc;
+    }
+    return SCAR_OK;
+}
+
+int scar_ckpt_load_stored(scar_ctx *c, int fd) {
+    if (!c || fd < 0) return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc == SCAR_OK) rc = ensure_stage(c);
+    if (rc != SCAR_OK) return rc;
+    const uint64_t bytes = c->g.n_elems * 4;
+    char *z = static_cast<char *>(c->z);
+    for (uint64_t off = 0; off < bytes; off += kIoStageBytes) {
+        const size_t n = (size_t)(bytes - off < kIoStageBytes ? bytes - off : kIoStageBytes);
+        if ((rc = read_all(fd, c->io_stage, n, off)) != SCAR_OK) return rc;
+        CU_TRY(cudaMemcpyAsync(z + off, c->io_stage, n, cudaMemcpyHostToDevice, c->stream));
+        CU_TRY(cudaStreamSynchronize(c->stream));  // the staging buffer is reused by the next chunk
+    }
+    return SCAR_OK;
+}
+
+int scar_ckpt_store_drained(scar_ctx *c, uint64_t ticket, int fd) {
+    if (!c || fd < 0) return SCAR_ERR_INVALID_ARG;
+    DrainSlot *sl = c->drain ? slot_of(c, ticket) : nullptr;
+    if (!sl) return SCAR_ERR_STATE;
+    CU_TRY(cudaEventSynchronize(sl->drained));
+    sl->state = 3;
+    if (sl->h_info->error) return SCAR_ERR_TIMEOUT;
+    const uint64_t k = sl->h_info->k;
+    const char *payload = static_cast<const char *>(sl->h_payload);
+    // Runs of consecutive block ids are contiguous both in the payload and in the file: one write per run.
+    uint64_t j = 0;
+    while (j < k) {
+        uint64_t e = j;
+        while (e + 1 < k && sl->h_sel[e + 1] == sl->h_sel[e] + 1) ++e;
+        uint64_t beg, len;
+        host_range(c, sl->h_sel[j], beg, len);
+        const uint64_t n_elems = sl->h_poff[e + 1] - sl->h_poff[j];
+        const int rc = write_all(fd, payload + sl->h_poff[j] * 4, (size_t)n_elems * 4, beg * 4);
+        if (rc != SCAR_OK) return rc;
+        j = e + 1;
+    }
+    return SCAR_OK;
+}
+
 int scar_ckpt_load(scar_ctx *c, const void *d_z_src) {
     if (!c || (!d_z_src && c->g.n_elems)) return SCAR_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(d_z_src) & 15) return SCAR_ERR_INVALID_ARG;
@@ -1175,6 +1300,7 @@ const char *scar_strerror(int code) {
         case SCAR_ERR_STATE: return "call not valid in this state";
         case SCAR_ERR_TIMEOUT: return "a bounded device-side wait gave up";
         case SCAR_ERR_CAPACITY: return "problem exceeds a fixed-size internal buffer";
+        case SCAR_ERR_IO: return "reading or writing the stored checkpoint failed";
         default: return "unknown error";
     }
 }
