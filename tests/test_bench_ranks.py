@@ -83,4 +83,5 @@ def test_save_byte_model():
 
     n = 1 << 30
     assert bench.save_bytes(n, 0) == 2 * n * 4
-    assert bench.save_bytes(n, n) == 5 * n * 4  # r = 1: (2 + 3r) N s
+    assert bench.save_bytes(n, n // 2) == (2 * n + 3 * (n // 2)) * 4  # (2 + 3r) N s
+    assert bench.save_bytes(n, n) == 4 * n * 4  # a full checkpoint is one fused pass: no second read
