@@ -207,34 +207,72 @@ def run_reference(args):
         t_all += b
     value = len(w.r_values) * 2 * n * ELEM * args.steps / t_save / 1e9
     sample = f"{n} of {full} elements ({w.n_blocks} blocks), numpy-generated with the same recipe"
+    nproc, model = host_cpu()
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_all / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64" if w.dtype == "f32" else "int64", "data": "synthetic",
-        "config": {"workload": DESCRIPTIONS[args.workload], "n_elems": n, "sample_of": full},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "config": {"workload": DESCRIPTIONS[args.workload] + (f" [sample: {n} of {full} elements]" if n != full else ""),
+                   "n_elems": n, "sample_of": full},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample, "nproc": nproc,
+                         "cpu_model": model},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
 
 
+def host_cpu():
+    """(logical cores, model string) of the host."""
+    model = "unknown"
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return os.cpu_count() or 1, model
+
+
+def time_oracle_steps(x, z, boff, lost_blocks, r_sweep, budget_s=5.0, max_reps=50):
+    """Repeats the oracle step until a few seconds of saves have been timed; (GB/s scanned, reps, seconds)."""
+    reps, t_save = 0, 0.0
+    while reps < 1 or (t_save < budget_s and reps < max_reps):
+        t_save += oracle_step(x, z, boff, lost_blocks, r_sweep)[0]
+        reps += 1
+    return reps * len(r_sweep) * 2 * x.size * ELEM / t_save / 1e9, reps, t_save
+
+
 def cpu_baseline(x_dev, z_dev, geom, lost_blocks, r_sweep):
-    """Times one oracle step on the device-resident workload (copied to the host), single thread."""
+    """Times the oracle on the device-resident workload (copied to the host): as it stands on one thread, and the
+    same source built with OpenMP (loops over blocks in parallel, the selection still the serial sort) on all
+    cores.  The headline `value` is the single-thread leg, the oracle exactly as the parity tests use it."""
+    import oracle
     from workloads import block_offsets
 
     x = x_dev.cpu().numpy()
     z = z_dev.cpu().numpy()
     boff = block_offsets(geom)
-    reps, t_save = 0, 0.0
-    while reps < 1 or (t_save < 5.0 and reps < 50):  # small sets: repeat until a few seconds have been timed
-        t_save += oracle_step(x, z, boff, lost_blocks, r_sweep)[0]
-        reps += 1
-    return {"value": reps * len(r_sweep) * 2 * x.size * ELEM / t_save / 1e9, "unit": UNIT, "cores": 1,
-            "kind": "oracle",
-            "sample": f"{reps} step(s) on all {x.size} elements ({geom.n_blocks} blocks) of the same buffers, "
-                      f"single thread, {t_save:.1f} s in saves"}
+    nproc, model = host_cpu()
+    what = f"all {x.size} elements ({geom.n_blocks} blocks) of the same buffers"
+    v1, reps1, t1 = time_oracle_steps(x, z, boff, lost_blocks, r_sweep)
+    legs = {"single_thread": {"value": v1, "unit": UNIT, "cores": 1, "sample": f"{reps1} step(s) on {what}, {t1:.1f} s in saves"}}
+    try:
+        threads = oracle.use_openmp(True)
+        oracle_step(x, z, boff, lost_blocks, r_sweep)  # first touch by the thread pool, untimed
+        vn, repsn, tn = time_oracle_steps(x, z, boff, lost_blocks, r_sweep)
+        legs["all_cores"] = {"value": vn, "unit": UNIT, "cores": threads,
+                             "sample": f"{repsn} step(s) on {what}, {tn:.1f} s in saves; OpenMP build of the same "
+                                       "source, selection serial"}
+    except Exception as e:  # no OpenMP runtime on the host: say so, keep the single-thread leg
+        legs["all_cores"] = {"unavailable": str(e)[:200]}
+    finally:
+        oracle.use_openmp(False)
+    return {"value": v1, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": legs["single_thread"]["sample"],
+            "nproc": nproc, "cpu_model": model, **legs}
 
 
 # ----------------------------------------------------------------------------- GPU arm
@@ -273,34 +311,25 @@ def device_workload(name, n_elems, rank, dev):
             w.lost_blocks)
 
 
-def run_gpu(args):
+class Measured:
+    """Raw results of the timed steps of one workload on this rank."""
+
+
+def measure_workload(api, name, n_elems, rank, dev, steps, warmup, barrier):
+    """W warm-up steps, then `steps` timed steps of the whole hot path over one synthetic parameter set, each
+    call bracketed by CUDA events on the stream the library launches on; then the per-phase durations through
+    the library's own events.  Returns a Measured holding the context and the buffers (the caller frees them)."""
     import torch
-    import torch.distributed as dist
 
-    from paper_1810_07354_b200 import api
-
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback for the library")
-    api.load_library()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    geom, z0, x0, r_sweep, lost_shards, lost_blocks = device_workload(args.workload, args.n_elems, rank, dev)
-    n = x0.numel()
-    x = x0.clone()
-    ck = api.ScarCheckpoint(x, n_shards=geom.n_shards, row_elems=geom.row_elems, block_elems=geom.block_elems)
+    m = Measured()
+    m.name = name
+    geom, z0, x0, r_sweep, lost_shards, lost_blocks = device_workload(name, n_elems, rank, dev)
+    m.geom, m.z0, m.x0, m.r_sweep, m.lost_shards, m.lost_blocks = geom, z0, x0, r_sweep, lost_shards, lost_blocks
+    m.n = x0.numel()
+    m.x = x0.clone()
+    m.ck = ck = api.ScarCheckpoint(m.x, n_shards=geom.n_shards, row_elems=geom.row_elems, block_elems=geom.block_elems)
     ctx = ck.ctx
-    nb = ck.n_blocks
+    m.nb = ck.n_blocks
     d_lost = torch.from_numpy(lost_blocks).to(dev) if lost_blocks is not None else None
 
     def recover(sync=False):
@@ -308,8 +337,8 @@ def run_gpu(args):
             return ck.recover_partial_blocks(d_lost, sync=sync)
         return ck.recover_partial(lost_shards, sync=sync)
 
-    z_lib = ck.views()["z"]  # the library's running checkpoint, aliased (no copy)
-    flush = torch.empty(64 << 20, dtype=torch.float32, device=dev)  # 256 MiB, larger than the 126 MB L2
+    m.z_lib = z_lib = ck.views()["z"]  # the library's running checkpoint, aliased (no copy)
+    m.flush = flush = torch.empty(64 << 20, dtype=torch.float32, device=dev)  # 256 MiB, larger than the 126 MB L2
 
     def reset_checkpoint():
         """Pristine running checkpoint, then an L2 flush; plain torch copies, outside every timed interval."""
@@ -317,10 +346,10 @@ def run_gpu(args):
         flush.zero_()
 
     def reset_live():
-        x.copy_(x0)
+        m.x.copy_(x0)
         flush.zero_()
 
-    lost_elems = int(recover(sync=True).lost_elems)
+    m.lost_elems = int(recover(sync=True).lost_elems)
     reset_live()
 
     ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
@@ -348,54 +377,108 @@ def run_gpu(args):
         rec.append((("recover", None), a, b))
         reset_live()  # put the live parameters back (not timed)
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         one_step([])
     barrier()
 
     # payload sizes per r (data dependent but fixed for this workload)
-    payload_elems = {}
+    m.payload_elems = {}
     for r in r_sweep:
         reset_checkpoint()
-        payload_elems[r] = int(ck.priority_save(r).payload_elems)
+        m.payload_elems[r] = int(ck.priority_save(r).payload_elems)
     barrier()
 
     # ---- timed region: K steps, device-timed
-    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid)) if rank == 0 else None
     launches0 = api.scar_ckpt_launch_count(ctx)
     rec = []
     barrier()
-    w0 = time.time()
-    for _ in range(args.steps):
+    m.w0 = time.time()
+    for _ in range(steps):
         one_step(rec)
     barrier()
-    w1 = time.time()
-    launches = api.scar_ckpt_launch_count(ctx) - launches0
-    clocks = sampler.stop(w0, w1) if sampler else None
-
-    t = {}
+    m.w1 = time.time()
+    m.launches = api.scar_ckpt_launch_count(ctx) - launches0
+    m.t = {}
     for (kind, r), a, b in rec:
-        t.setdefault((kind, r), []).append(a.elapsed_time(b))
-    tot_ms = sum(sum(v) for v in t.values())
-    save_ms = sum(sum(v) for (kind, _), v in t.items() if kind == "save")
-    tot_ms, save_ms = max_over_ranks([tot_ms, save_ms], dev, world)
+        m.t.setdefault((kind, r), []).append(a.elapsed_time(b))
 
-    # ---- dominant kernel (block scores) timed live through the library's own stream events
+    # ---- phases (and with them the dominant kernel, block scores) timed live through the library's own
+    # stream events
     api.scar_ckpt_profile(ctx, True)
-    phase = {r: [] for r in r_sweep}
-    rec_phase = []
-    for _ in range(min(args.steps, 10)):
+    m.phase = {r: [] for r in r_sweep}
+    m.rec_phase = []
+    for _ in range(min(steps, 10)):
         for r in r_sweep:
             reset_checkpoint()
             ck.priority_save(r, sync=False)
-            phase[r].append(api.scar_ckpt_profile_read(ctx))
+            m.phase[r].append(api.scar_ckpt_profile_read(ctx))
         flush.zero_()
         recover()
-        rec_phase.append(api.scar_ckpt_profile_read(ctx))
+        m.rec_phase.append(api.scar_ckpt_profile_read(ctx))
         reset_live()
     api.scar_ckpt_profile(ctx, False)
     # the scoring kernel runs on its own in every save that is not a full checkpoint (those fuse it with the pack)
-    partial = [r for r in r_sweep if payload_elems[r] < n] or list(r_sweep)
-    score_ms = float(np.mean([p[0] for r in partial for p in phase[r]]))
+    partial = [r for r in r_sweep if m.payload_elems[r] < m.n] or list(r_sweep)
+    m.score_ms = float(np.mean([p[0] for r in partial for p in m.phase[r]]))
+    return m
+
+
+def summarise(m, peak):
+    """Per-r save figures, norm and recovery figures of one measured workload."""
+    scanned = 2 * m.n * ELEM
+    per_r = {}
+    for r in m.r_sweep:
+        ms = float(np.median(m.t[("save", r)]))
+        by = save_bytes(m.n, m.payload_elems[r])
+        ph = np.median(np.array(m.phase[r]), axis=0)
+        per_r[str(r)] = {"save_ms": ms, "save_ms_min": float(np.min(m.t[("save", r)])), "scanned_gbs": scanned / ms / 1e6,
+                         "algorithmic_gbs": by / ms / 1e6, "frac_of_measured_peak": by / ms / 1e6 / peak,
+                         "frac_of_8tbs": by / ms / 1e6 / 8000.0, "blocks_per_s": m.nb / (ms * 1e-3),
+                         "payload_elems": m.payload_elems[r],
+                         "phase_ms": {"scores": float(ph[0]), "select": float(ph[1]), "pack": float(ph[2])}}
+    norm_ms = float(np.median(m.t[("norm", None)]))
+    rec_ms = float(np.median(m.t[("recover", None)]))
+    rph = np.median(np.array(m.rec_phase), axis=0)
+    rec_gbs = 3 * m.lost_elems * ELEM / rec_ms / 1e6
+    return {
+        "per_r": per_r,
+        "perturbation_norm": {"ms": norm_ms, "gbs": scanned / norm_ms / 1e6, "frac_of_measured_peak": scanned / norm_ms / 1e6 / peak},
+        "partial_recovery": {"ms": rec_ms, "gbs": rec_gbs, "frac_of_measured_peak": rec_gbs / peak,
+                             "lost_elems": m.lost_elems, "phase_ms": {"restore_and_norm": float(rph[3])}},
+        "block_scores": {"ms": m.score_ms, "gbs": scanned / m.score_ms / 1e6, "frac_of_measured_peak": scanned / m.score_ms / 1e6 / peak},
+    }
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_1810_07354_b200 import api
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback for the library")
+    api.load_library()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid)) if rank == 0 else None
+    m = measure_workload(api, args.workload, args.n_elems, rank, dev, args.steps, args.warmup, barrier)
+    clocks = sampler.stop(m.w0, m.w1) if sampler else None
+    n, nb, r_sweep = m.n, m.nb, m.r_sweep
+
+    tot_ms = sum(sum(v) for v in m.t.values())
+    save_ms = sum(sum(v) for (kind, _), v in m.t.items() if kind == "save")
+    tot_ms, save_ms = max_over_ranks([tot_ms, save_ms], dev, world)
 
     if rank != 0:
         barrier()
@@ -406,58 +489,61 @@ def run_gpu(args):
     peak, peak_kind = hbm_peak()
     scanned = 2 * n * ELEM
     value = job_throughput_gbs(world, len(r_sweep) * scanned * args.steps, save_ms)
-    per_r = {}
-    for r in r_sweep:
-        ms = float(np.median(t[("save", r)]))
-        by = save_bytes(n, payload_elems[r])
-        ph = np.median(np.array(phase[r]), axis=0)
-        per_r[str(r)] = {"save_ms": ms, "save_ms_min": float(np.min(t[("save", r)])), "scanned_gbs": scanned / ms / 1e6, "algorithmic_gbs": by / ms / 1e6,
-                         "frac_of_measured_peak": by / ms / 1e6 / peak, "frac_of_8tbs": by / ms / 1e6 / 8000.0,
-                         "blocks_per_s": nb / (ms * 1e-3), "payload_elems": payload_elems[r],
-                         "phase_ms": {"scores": float(ph[0]), "select": float(ph[1]), "pack": float(ph[2])}}
-    norm_ms = float(np.median(t[("norm", None)]))
-    rec_ms = float(np.median(t[("recover", None)]))
-    rph = np.median(np.array(rec_phase), axis=0)
-    achieved = scanned / (score_ms * 1e-3) / 1e9
+    summ = summarise(m, peak)
+    achieved = scanned / (m.score_ms * 1e-3) / 1e9
     l2_note = ("inputs larger than L2; " if scanned > (512 << 20) else "inputs NOT larger than L2; ") + \
         "L2 flushed by a 256 MiB write after every untimed state reset and before every timed call"
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": tot_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32" if x0.dtype == torch.float32 else "int32", "data": "synthetic",
+        "dtype": "f32" if m.x0.dtype == torch.float32 else "int32", "data": "synthetic",
         "config": {"workload": DESCRIPTIONS[args.workload], "n_elems": n, "n_blocks": nb, "r_sweep": list(r_sweep),
                    "l2": l2_note, "value_is": "sum over the r sweep of 2*N*4 bytes / sum of save times",
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
         "save_ms_per_step": save_ms / args.steps,
-        "per_r": per_r,
-        "perturbation_norm": {"ms": norm_ms, "gbs": scanned / norm_ms / 1e6},
-        "partial_recovery": {"ms": rec_ms, "gbs": 3 * lost_elems * ELEM / rec_ms / 1e6, "lost_elems": lost_elems,
-                             "phase_ms": {"restore": float(rph[3]), "reduce": float(rph[4])}},
+        "per_r": summ["per_r"],
+        "perturbation_norm": summ["perturbation_norm"],
+        "partial_recovery": summ["partial_recovery"],
         "roofline": {"bound": "hbm", "kernel": "k_block_scores", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": f"of {peak_kind}",
                      "traffic": recorded_traffic(n) if args.workload == "cnn" else None,
-                     "bytes_per_launch": scanned, "ms_per_launch": score_ms},
-        "gpu_launches": int(launches),
+                     "bytes_per_launch": scanned, "ms_per_launch": m.score_ms},
+        "gpu_launches": int(m.launches),
         "clocks": clocks,
-        "wall_s_timed_region": w1 - w0,
+        "wall_s_timed_region": m.w1 - m.w0,
     }
 
     if not args.no_e2e:
-        line["e2e"] = run_e2e(api, ck, x0, z_lib, z0, r_sweep, lost_shards, lost_elems, n, nb, world, flush)
+        line["e2e"] = run_e2e(api, m.ck, m.x0, m.z_lib, m.z0, r_sweep, m.lost_shards, m.lost_elems, n, nb, world, m.flush)
     if world == 1 and not args.no_cpu_baseline:
-        if lost_blocks is None:
+        if m.lost_blocks is None:
             from workloads import shard_block_ranges
 
             lb = np.zeros(nb, dtype=np.uint8)
-            for lo, hi in shard_block_ranges(nb, geom.n_shards)[np.flatnonzero(lost_shards)]:
+            for lo, hi in shard_block_ranges(nb, m.geom.n_shards)[np.flatnonzero(m.lost_shards)]:
                 lb[lo:hi] = 1
         else:
-            lb = lost_blocks
-        line["cpu_baseline"] = cpu_baseline(x0, z0, geom, lb, r_sweep)
+            lb = m.lost_blocks
+        line["cpu_baseline"] = cpu_baseline(m.x0, m.z0, m.geom, lb, r_sweep)
     if world == 1 and not args.no_extras:
-        line["extras"] = run_extras(api, ck, x, x0, z_lib, z0, geom, r_sweep, flush, dev,
+        line["extras"] = run_extras(api, m.ck, m.x, m.x0, m.z_lib, m.z0, m.geom, r_sweep, m.flush, dev,
                                     with_bylayer=args.workload == "cnn" and n >= (1 << 28))
+    if world == 1 and args.workload == "cnn" and not args.no_configs:
+        # The other four parameter sets (far smaller: their steps take a fraction of a millisecond) measured the
+        # same way, after the headline's buffers are gone; same keys per set, fewer steps.
+        configs = {"cnn": summ}
+        m.ck.close()
+        del m
+        torch.cuda.empty_cache()
+        for name in ("tiny", "mlr", "mf", "lda"):
+            mm = measure_workload(api, name, 0, rank, dev, min(args.steps, 20), max(args.warmup, 3), barrier)
+            configs[name] = dict(summarise(mm, peak), n_elems=mm.n, n_blocks=mm.nb, workload=DESCRIPTIONS[name],
+                                 gpu_launches=int(mm.launches))
+            mm.ck.close()
+            del mm
+            torch.cuda.empty_cache()
+        line["configs"] = configs
     print(json.dumps(line))
     barrier()
     if world > 1:
@@ -628,6 +714,8 @@ def main():
                     help="elements of the CNN-scale parameter vector (default 2**30)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="with the default workload: skip the measurement of the four smaller parameter sets")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the measurements beside the headline step (baseline selectors, drain, by-layer layout)")
     args = ap.parse_args()

@@ -346,6 +346,19 @@ double scar_irreducible_error(double delta_max, double c);
  * SCAR_ERR_STATE on an empty buffer. */
 int scar_ckpt_selftest_arm_timeout(scar_ctx *ctx);
 
+/* Diagnostic builds only (library compiled with -DSCAR_SELECT_STAMPS; otherwise
+ * SCAR_ERR_STATE).  Waits for the stream and copies the 32 time stamps of the
+ * most recent selection kernel: SM clock cycles of its first CTA at
+ *   [0] start, [1] keys loaded, then for digit pass p = 0..5
+ *   [2+4p] shared histogram built, [3+4p] flushed to the global histogram,
+ *   [4+4p] every CTA has arrived, [5+4p] digit resolved,
+ *   [26] own counts known, [27] every CTA's record read, [28] output bases
+ *   known, [29] ids and offsets written.
+ * Stamps of passes that did not run keep the value of an earlier selection (or
+ * zero).  No counterpart in the paper: it shows where the selection of
+ * checkpoint step 3 spends its time. */
+int scar_ckpt_debug_select_stamps(scar_ctx *ctx, int64_t stamps[32]);
+
 /* Waits for the stream, frees everything the context owns (never x). */
 int scar_ckpt_destroy(scar_ctx *ctx);
 

@@ -23,32 +23,50 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "scar_oracle.c")
 _SO = os.path.join(_HERE, "liboracle.so")
+_SO_OMP = os.path.join(_HERE, "liboracle_omp.so")
 _lock = threading.Lock()
 _lib = None
+_lib_omp = None
 
 
-def build(force: bool = False) -> str:
-    """Compile ``scar_oracle.c`` with gcc (strict IEEE: no contraction, no fast-math)."""
-    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
-        tmp = f"{_SO}.{os.getpid()}.tmp"
+def build(force: bool = False, openmp: bool = False) -> str:
+    """Compile ``scar_oracle.c`` with gcc (strict IEEE: no contraction, no fast-math).
+
+    ``openmp``: the second build of the same file (``-fopenmp``) whose loops over blocks run on all host cores.
+    It exists only to be timed as the all-core CPU baseline; pins and parity tests use the plain build."""
+    so = _SO_OMP if openmp else _SO
+    if force or not os.path.exists(so) or os.path.getmtime(so) < os.path.getmtime(_SRC):
+        tmp = f"{so}.{os.getpid()}.tmp"
         subprocess.check_call(
-            ["gcc", "-O2", "-ffp-contract=off", "-std=c99", "-Wall", "-Wextra", "-fPIC", "-shared",
-             "-o", tmp, _SRC, "-lm"]
+            ["gcc", "-O2", "-ffp-contract=off", "-std=c99", "-Wall", "-Wextra", "-fPIC", "-shared"]
+            + (["-fopenmp"] if openmp else []) + ["-o", tmp, _SRC, "-lm"]
         )
-        os.replace(tmp, _SO)
-    return _SO
+        os.replace(tmp, so)
+    return so
 
 
 _u64, _i64, _dbl, _int = C.c_uint64, C.c_int64, C.c_double, C.c_int
 _p = C.c_void_p
 
 
+_use_openmp = False
+
+
+def use_openmp(on: bool) -> int:
+    """Switches every later call of this package between the plain build and the OpenMP build of the same
+    source (for timing the all-core baseline only); returns the number of threads the chosen build uses."""
+    global _use_openmp
+    _use_openmp = bool(on)
+    return int(_load().scar_oracle_threads())
+
+
 def _load():
-    global _lib
+    global _lib, _lib_omp
     with _lock:
-        if _lib is None:
-            lib = C.CDLL(build())
+        if (_lib_omp if _use_openmp else _lib) is None:
+            lib = C.CDLL(build(openmp=_use_openmp))
             sig = {
+                "scar_oracle_threads": (_int, []),
                 "scar_oracle_count_blocks": (_u64, [_u64, _u64, _u64]),
                 "scar_oracle_layout_offsets": (None, [_u64, _u64, _u64, _p]),
                 "scar_oracle_expand_shards": (None, [_u64, _u64, _p, _p]),
@@ -66,8 +84,11 @@ def _load():
             for name, (res, args) in sig.items():
                 fn = getattr(lib, name)
                 fn.restype, fn.argtypes = res, args
-            _lib = lib
-    return _lib
+            if _use_openmp:
+                _lib_omp = lib
+            else:
+                _lib = lib
+    return _lib_omp if _use_openmp else _lib
 
 
 def _ptr(a: Optional[np.ndarray]):

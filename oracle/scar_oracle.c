@@ -13,6 +13,12 @@
  * ascending element order, integer sums in 64-bit integers.  There is no
  * blocking, vectorisation or reordering.
  *
+ * The same file also builds with -fopenmp, only to time the oracle on all host
+ * cores: the loops over blocks (scores, pack, cache update, recovery) then run
+ * in parallel, the selection stays the serial sort.  Per-block sums keep their
+ * element order either way; only the recovery's sum ACROSS blocks changes its
+ * order in that build.  Every pin and every parity test uses the plain build.
+ *
  * Notation follows the paper's appendix proof of Theorem 4.1:
  *   x = live parameters x^(T), z = running checkpoint, S = lost set.
  * A "parameter" for distance, selection and loss is one block of contiguous
@@ -24,6 +30,18 @@
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#define SCAR_PRAGMA(x) _Pragma(#x)
+#define SCAR_OVER_BLOCKS SCAR_PRAGMA(omp parallel for schedule(static))
+#define SCAR_OVER_BLOCKS_SUM(...) SCAR_PRAGMA(omp parallel for schedule(static) reduction(+ : __VA_ARGS__))
+int scar_oracle_threads(void) { return omp_get_max_threads(); }
+#else
+#define SCAR_OVER_BLOCKS
+#define SCAR_OVER_BLOCKS_SUM(...)
+int scar_oracle_threads(void) { return 1; }
+#endif
 
 /* ---- geometry ----------------------------------------------------------- */
 
@@ -73,6 +91,7 @@ void scar_oracle_expand_shards(uint64_t n_blocks, uint64_t n_shards, const uint8
 void scar_oracle_scores_f32(const float *x, const float *z, const uint64_t *boff, uint64_t n_blocks,
                             double *score)
 {
+    SCAR_OVER_BLOCKS
     for (uint64_t b = 0; b < n_blocks; ++b) {
         double acc = 0.0;
         for (uint64_t i = boff[b]; i < boff[b + 1]; ++i) {
@@ -89,6 +108,7 @@ void scar_oracle_scores_f32(const float *x, const float *z, const uint64_t *boff
 void scar_oracle_scores_f32_l1(const float *x, const float *z, const uint64_t *boff, uint64_t n_blocks,
                                double *score)
 {
+    SCAR_OVER_BLOCKS
     for (uint64_t b = 0; b < n_blocks; ++b) {
         double acc = 0.0;
         for (uint64_t i = boff[b]; i < boff[b + 1]; ++i)
@@ -103,6 +123,7 @@ void scar_oracle_scores_f32_l1(const float *x, const float *z, const uint64_t *b
 void scar_oracle_scores_i32(const int32_t *x, const int32_t *z, const uint64_t *boff, uint64_t n_blocks,
                             uint64_t *score)
 {
+    SCAR_OVER_BLOCKS
     for (uint64_t b = 0; b < n_blocks; ++b) {
         uint64_t acc = 0;
         for (uint64_t i = boff[b]; i < boff[b + 1]; ++i) {
@@ -201,17 +222,22 @@ void scar_oracle_pack(const uint32_t *x, const uint64_t *boff, const uint32_t *s
 {
     uint64_t out = 0;
     for (uint64_t j = 0; j < k; ++j) {
-        uint64_t b = sel[j];
         poff[j] = out;
-        for (uint64_t i = boff[b]; i < boff[b + 1]; ++i) payload[out++] = x[i];
+        out += boff[sel[j] + 1] - boff[sel[j]];
     }
     poff[k] = out;
+    SCAR_OVER_BLOCKS
+    for (uint64_t j = 0; j < k; ++j) {
+        uint64_t b = sel[j], at = poff[j];
+        for (uint64_t i = boff[b]; i < boff[b + 1]; ++i) payload[at++] = x[i];
+    }
 }
 
 /* Section 4.3 step 4, the cache refresh: z_b := x_b bytewise for
  * every selected block; all other blocks of z keep their bytes. */
 void scar_oracle_update(uint32_t *z, const uint32_t *x, const uint64_t *boff, const uint32_t *sel, uint64_t k)
 {
+    SCAR_OVER_BLOCKS
     for (uint64_t j = 0; j < k; ++j) {
         uint64_t b = sel[j];
         for (uint64_t i = boff[b]; i < boff[b + 1]; ++i) z[i] = x[i];
@@ -232,6 +258,7 @@ double scar_oracle_recover_f32(float *x, const float *z, const uint64_t *boff, u
 {
     double acc = 0.0;
     uint64_t nb = 0, ne = 0;
+    SCAR_OVER_BLOCKS_SUM(acc, nb, ne)
     for (uint64_t b = 0; b < n_blocks; ++b) {
         if (lost_blocks && !lost_blocks[b]) continue;
         ++nb;
@@ -242,6 +269,7 @@ double scar_oracle_recover_f32(float *x, const float *z, const uint64_t *boff, u
         }
     }
     if (write)
+        SCAR_OVER_BLOCKS
         for (uint64_t b = 0; b < n_blocks; ++b) {
             if (lost_blocks && !lost_blocks[b]) continue;
             memcpy(x + boff[b], z + boff[b], (boff[b + 1] - boff[b]) * sizeof(float));
@@ -257,6 +285,7 @@ uint64_t scar_oracle_recover_i32(int32_t *x, const int32_t *z, const uint64_t *b
                                  uint64_t *n_lost_elems)
 {
     uint64_t acc = 0, nb = 0, ne = 0;
+    SCAR_OVER_BLOCKS_SUM(acc, nb, ne)
     for (uint64_t b = 0; b < n_blocks; ++b) {
         if (lost_blocks && !lost_blocks[b]) continue;
         ++nb;
@@ -267,6 +296,7 @@ uint64_t scar_oracle_recover_i32(int32_t *x, const int32_t *z, const uint64_t *b
         }
     }
     if (write)
+        SCAR_OVER_BLOCKS
         for (uint64_t b = 0; b < n_blocks; ++b) {
             if (lost_blocks && !lost_blocks[b]) continue;
             memcpy(x + boff[b], z + boff[b], (boff[b + 1] - boff[b]) * sizeof(int32_t));

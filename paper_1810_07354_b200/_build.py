@@ -26,9 +26,12 @@ def is_stale() -> bool:
     return any(os.path.getmtime(s) > t for s in _sources())
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile ``csrc/*.cu`` into ``libscar.so`` next to this file if it is missing or out of date."""
-    if not force and not is_stale():
+def build(force: bool = False, verbose: bool = False, select_stamps: bool = False) -> str:
+    """Compile ``csrc/*.cu`` into ``libscar.so`` next to this file if it is missing or out of date.
+
+    ``select_stamps``: diagnostic build whose selection kernel records cycle stamps of its phases
+    (``scar_ckpt_debug_select_stamps``); rebuild without it for measurements."""
+    if not force and not select_stamps and not is_stale():
         return LIB
     nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
     if not os.path.exists(nvcc):
@@ -36,8 +39,16 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = f"{LIB}.{os.getpid()}.tmp"
     units = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cu"))
     cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-o", tmp, *units]
+    if select_stamps:
+        cmd += ["-DSCAR_SELECT_STAMPS"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)
     return LIB
+
+
+if __name__ == "__main__":
+    import sys
+
+    print(build(force=True, verbose="-v" in sys.argv, select_stamps="--select-stamps" in sys.argv))

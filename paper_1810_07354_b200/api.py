@@ -96,6 +96,7 @@ _SIGS = {
     "scar_iteration_cost_bound": (_dbl, [_dbl, _dbl, _dbl]),
     "scar_irreducible_error": (_dbl, [_dbl, _dbl]),
     "scar_ckpt_selftest_arm_timeout": (_int, [_vp]),
+    "scar_ckpt_debug_select_stamps": (_int, [_vp, C.POINTER(C.c_int64)]),
     "scar_ckpt_destroy": (_int, [_vp]),
     "scar_strerror": (C.c_char_p, [_int]),
 }
@@ -365,6 +366,13 @@ def scar_irreducible_error(delta_max: float, c: float) -> float:
 
 def scar_ckpt_selftest_arm_timeout(ctx: int) -> None:
     _check(load_library().scar_ckpt_selftest_arm_timeout(ctx), "scar_ckpt_selftest_arm_timeout")
+
+
+def scar_ckpt_debug_select_stamps(ctx: int) -> list:
+    """Cycle stamps of the last selection kernel (diagnostic builds of the library only)."""
+    st = (C.c_int64 * 32)()
+    _check(load_library().scar_ckpt_debug_select_stamps(ctx, st), "scar_ckpt_debug_select_stamps")
+    return list(st)
 
 
 def scar_ckpt_destroy(ctx: int) -> None:

@@ -13,6 +13,7 @@
 #include <type_traits>
 
 #include "geom.cuh"
+#include "sel_state.cuh"
 
 namespace scar {
 
@@ -86,6 +87,12 @@ __device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.
 template <typename V> __device__ __forceinline__ V ld_stream(const V *p) { return __ldcs(p); }
 template <typename V> __device__ __forceinline__ void st_stream(V *p, const V &v) { __stcs(p, v); }
 
+// Keeps the compiler from moving a store above a load that precedes it in the source.  In the restoring pass a
+// batch's stores depend on its loads; when the compiler interleaves them to save registers ("load, store, load,
+// store"), each load waits behind a store that waits for the load before it, and a batch costs four round
+// trips to memory instead of one (measured: a 3x slower pass, depending on what else the kernel contained).
+__device__ __forceinline__ void loads_before_stores() { asm volatile("" ::: "memory"); }
+
 template <int G, typename W> __device__ __forceinline__ W group_sum(W v) {
 #pragma unroll
     for (int o = G / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -94,17 +101,25 @@ template <int G, typename W> __device__ __forceinline__ W group_sum(W v) {
 
 // One batch = four units (16-byte vectors, or single elements on the
 // element-wise path) per stream and lane, G units apart.  Units past the end of
-// the block load as zero, which adds nothing to either distance.
+// the block count as zero, which adds nothing to either distance.  Requires
+// n > 0.  The loads themselves are unconditional (a unit past the end reads the
+// block's last unit instead and the value is dropped): eight loads in one
+// straight line are issued back to back, whereas loads under eight branches
+// were, in some builds, each waited for before the next was issued, which made
+// a pass over short blocks three times slower.
 template <typename U, int G>
 __device__ __forceinline__ void load_batch(const U *__restrict__ xs, const U *__restrict__ zs, uint64_t u, uint64_t n,
                                            U (&xr)[4], U (&zr)[4]) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const uint64_t i = u + (uint64_t)j * G;
-        if (i < n) {
-            xr[j] = ld_stream(xs + i);
-            zr[j] = ld_stream(zs + i);
-        } else {
+        const uint64_t at = i < n ? i : n - 1;
+        xr[j] = ld_stream(xs + at);
+        zr[j] = ld_stream(zs + at);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if (u + (uint64_t)j * G >= n) {
             xr[j] = U{};
             zr[j] = U{};
         }
@@ -140,19 +155,27 @@ __device__ __forceinline__ typename Elem<T, NORM>::wide_t block_distance(T *__re
     U xc[4], zc[4], xn[4], zn[4];
     uint64_t u = lane;
     unsigned it = 0;
-    if (!WRITE) {
-        // Read-only pass: nothing can hold back the loads, so the plain loop is
-        // the faster form (full batches unguarded, then one guarded batch).  A
-        // batch counts as full only when it is full for every lane of the group,
-        // so the lanes of a group never diverge between the two forms.
+    if (!WRITE || G < 32) {
+        // Plain loop (full batches unguarded, then one guarded batch).  For the
+        // read-only pass nothing can hold back the loads, so this is the faster
+        // form.  It is also the form of the restoring pass over short blocks
+        // (G < 32: a block is about one batch, so there is no next batch to
+        // load ahead, and the registers of the pipelined form below would only
+        // cost occupancy: 16 resident warps per SM instead of 48).  A batch
+        // counts as full only when it is full for every lane of the group, so
+        // the lanes of a group never diverge between the two forms.
         for (; u - lane + step <= n; u += step) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 xc[j] = ld_stream(xs + u + (uint64_t)j * G);
                 zc[j] = ld_stream(zs + u + (uint64_t)j * G);
             }
+            if (WRITE) loads_before_stores();
 #pragma unroll
-            for (int j = 0; j < 4; ++j) E::addu(a[j], xc[j], zc[j]);
+            for (int j = 0; j < 4; ++j) {
+                E::addu(a[j], xc[j], zc[j]);
+                if (WRITE) st_stream(xs + u + (uint64_t)j * G, zc[j]);
+            }
             if (E::kFlush && (++it & kFlushMask) == 0) {
                 total += ((wide_t)a[0] + (wide_t)a[1]) + ((wide_t)a[2] + (wide_t)a[3]);
                 a[0] = a[1] = a[2] = a[3] = 0;
@@ -160,8 +183,12 @@ __device__ __forceinline__ typename Elem<T, NORM>::wide_t block_distance(T *__re
         }
         if (u < n) {
             load_batch<U, G>(xs, zs, u, n, xc, zc);
+            if (WRITE) loads_before_stores();
 #pragma unroll
-            for (int j = 0; j < 4; ++j) E::addu(a[j], xc[j], zc[j]);
+            for (int j = 0; j < 4; ++j) {
+                E::addu(a[j], xc[j], zc[j]);
+                if (WRITE && u + (uint64_t)j * G < n) st_stream(xs + u + (uint64_t)j * G, zc[j]);
+            }
         }
         total += ((wide_t)a[0] + (wide_t)a[1]) + ((wide_t)a[2] + (wide_t)a[3]);
         return group_sum<G, wide_t>(total);
@@ -195,8 +222,6 @@ __device__ __forceinline__ typename Elem<T, NORM>::wide_t block_distance(T *__re
 
 // ---- a1: score of every block ----------------------------------------------
 
-struct SelState;  // select.cuh
-
 // Block total -> stored score, times the block's weight when the caller set
 // weights (float data only; Appendix C: a positive combination of block norms
 // is still a norm).
@@ -207,12 +232,14 @@ __device__ __forceinline__ typename E::score_t weighted(typename E::wide_t s, co
     return (typename E::score_t)s;
 }
 
+// sel_state / info: the scoring pass is what runs before a selection, so its first CTAs clear the selection's
+// counters, histograms and records and the save's result record (both may be nullptr: nothing is cleared).
 template <typename T, int NORM, int G, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 k_block_scores(const T *__restrict__ x, const T *__restrict__ z, Geom g, const float *__restrict__ weight,
-               typename Elem<T, NORM>::score_t *__restrict__ score, unsigned long long *key_or, unsigned *hist0,
-               int hist0_len) {
+               typename Elem<T, NORM>::score_t *__restrict__ score, SelState *sel_state, SaveInfoDev *info) {
     using E = Elem<T, NORM>;
+    if (sel_state) sel_state_clear(sel_state, info);
     const int lane = threadIdx.x & (G - 1);
     const uint64_t grp = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
     const bool valid = grp < g.n_blocks;
@@ -222,69 +249,17 @@ k_block_scores(const T *__restrict__ x, const T *__restrict__ z, Geom g, const f
     if (valid && lane == 0) {
         typename E::score_t sc = weighted<E>(s, weight, grp);
         score[grp] = sc;
-        if (sizeof(typename E::score_t) == 8) {
+        if (sel_state && sizeof(typename E::score_t) == 8) {
             // Remember which key bits occur at all, so that radix passes over
             // digits that are zero in every key can be skipped.
             unsigned long long bits = (unsigned long long)sc;
-            unsigned long long seen = *reinterpret_cast<volatile unsigned long long *>(key_or);
-            if (bits & ~seen) atomicOr(key_or, bits);
+            unsigned long long seen = *reinterpret_cast<volatile unsigned long long *>(&sel_state->key_or);
+            if (bits & ~seen) atomicOr(&sel_state->key_or, bits);
         }
     }
-    // The first radix histogram is accumulated after this kernel; clear it here.
-    if (blockIdx.x == 0)
-        for (int i = threadIdx.x; i < hist0_len; i += kThreads) hist0[i] = 0;
 }
 
-// ---- a4 / a5: per-block perturbation over the lost set, optional restore ---
-
-template <typename T, int NORM, int G, bool VEC, bool WRITE>
-__global__ void __launch_bounds__(kThreads)
-k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S, const float *__restrict__ weight,
-                 typename Elem<T, NORM>::score_t *__restrict__ part) {
-    using E = Elem<T, NORM>;
-    griddep_launch();  // the reduction that follows may be scheduled early; it waits for this grid before reading
-    const int lane = threadIdx.x & (G - 1);
-    if (G < 32 && S.mode == 2) {
-        // Per-block mask with several blocks per warp: a warp takes 32 consecutive
-        // blocks, ballots which are lost and hands only those to its groups, so that
-        // a sparse mask does not leave most lanes idle.
-        constexpr int kGroups = 32 / G;
-        const int wl = threadIdx.x & 31, gi = wl / G;
-        const uint64_t b0 = (((uint64_t)blockIdx.x * kThreads + threadIdx.x) >> 5) * 32;
-        const bool lost = b0 + wl < g.n_blocks && S.mask[b0 + wl] != 0;
-        const unsigned bal = __ballot_sync(0xffffffffu, lost);
-        const int cnt = __popc(bal);
-        for (int t0 = 0; t0 < cnt; t0 += kGroups) {  // same trip count for every lane of the warp
-            const int t = t0 + gi;
-            const bool valid = t < cnt;
-            uint32_t b = 0;
-            uint64_t beg = 0, len = 0;
-            if (valid) {
-                b = (uint32_t)(b0 + __fns(bal, 0, t + 1));
-                g.range(b, beg, len);
-            }
-            typename E::wide_t s = block_distance<T, NORM, G, VEC, WRITE>(x, z, beg, len, lane);
-            if (valid && lane == 0) part[b] = weighted<E>(s, weight, b);
-        }
-        return;
-    }
-    const uint64_t w = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
-    uint32_t b = 0;
-    const bool valid = S.block_of(w, b);
-    uint64_t beg = 0, len = 0;
-    if (valid) g.range(b, beg, len);
-    typename E::wide_t s = block_distance<T, NORM, G, VEC, WRITE>(x, z, beg, len, lane);
-    if (valid && lane == 0) part[b] = weighted<E>(s, weight, b);
-}
-
-// Lost shards as a per-block mask, for lost sets with more runs than LostSet holds.
-static __global__ void __launch_bounds__(kThreads)
-k_expand_shards(Geom g, const uint8_t *__restrict__ shard_mask, uint8_t *__restrict__ block_mask) {
-    const uint64_t b = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (b < g.n_blocks) block_mask[b] = shard_mask[g.shard_of((uint32_t)b)] != 0;
-}
-
-// ---- final reduction of the per-block partials in a fixed order -------------
+// ---- final reduction of a recovery / norm pass, in a fixed order ------------------
 
 struct NormInfoDev {
     double l2;
@@ -292,9 +267,6 @@ struct NormInfoDev {
     unsigned long long lost_blocks;
     unsigned long long lost_elems;
 };
-
-constexpr int kReduceTile = 1024;  // work items per CTA in the reduction
-constexpr int kReducePer = kReduceTile / kThreads;
 
 template <typename W> __device__ __forceinline__ W cta_sum(W v, W *sh) {
     v = group_sum<32, W>(v);
@@ -308,72 +280,337 @@ template <typename W> __device__ __forceinline__ W cta_sum(W v, W *sh) {
     return t;
 }
 
-// Each CTA sums a fixed tile of per-block partials (fp64 for float data, exact
-// 64-bit for integer data) together with the lost block/element counts; the
-// CTA that finishes last adds the tile sums in tile order.  Which CTA is last
-// does not affect the order of any addition.
+// Scratch of the reduction: one slot per CTA of the pass and one per watcher.  A slot holds kSlotEmpty except
+// between its owner's store and the watcher's read, so the value itself tells the reader that it has arrived
+// (an aligned 8-byte store is seen whole or not at all); no fence, ticket or atomic is involved.
+constexpr unsigned long long kSlotEmpty = ~0ull;
+constexpr unsigned kMaxWatchers = kThreads;
+struct NormScratch {
+    unsigned long long *cta_val;     // per CTA: sum of its blocks' partials (bits of a double, or a uint64)
+    unsigned long long *cta_blocks;  // per CTA: lost blocks it covered
+    unsigned long long *cta_elems;   // per CTA: their elements
+    unsigned long long *tile_val;    // the same per watcher, kMaxWatchers of each
+    unsigned long long *tile_blocks;
+    unsigned long long *tile_elems;
+};
+// 8-byte words a launch of n_ctas CTAs needs: three arrays of n_ctas, then three of kMaxWatchers.
+inline size_t norm_scratch_words(uint64_t n_ctas) { return 3 * (size_t)n_ctas + 3 * kMaxWatchers; }
+inline NormScratch norm_scratch_at(unsigned long long *base, uint64_t n_ctas) {
+    NormScratch rs;
+    rs.cta_val = base;
+    rs.cta_blocks = base + n_ctas;
+    rs.cta_elems = base + 2 * n_ctas;
+    rs.tile_val = base + 3 * n_ctas;
+    rs.tile_blocks = rs.tile_val + kMaxWatchers;
+    rs.tile_elems = rs.tile_val + 2 * kMaxWatchers;
+    return rs;
+}
+
+// How many CTAs at the end of a grid add up the others' slots.
+__host__ __device__ inline unsigned norm_watchers(unsigned grid) {
+    const unsigned n = grid / 1024;
+    return n < 1 ? 1 : (n > kMaxWatchers ? kMaxWatchers : n);
+}
+
+constexpr unsigned kSlotSpinLimit = 1u << 20;  // a quarter of a second at the earliest
+
+__device__ __forceinline__ unsigned long long slot_peek(const unsigned long long *slot) {
+    return *reinterpret_cast<const volatile unsigned long long *>(slot);
+}
+// v: what slot_peek saw.  Waits (with a bound) until the slot's owner has filled it, and empties it again for the
+// next launch.  false: gave up.
+__device__ __forceinline__ bool slot_take(unsigned long long *slot, unsigned long long &v) {
+    volatile unsigned long long *p = slot;
+    unsigned tries = 0;
+    while (v == kSlotEmpty) {
+        if (++tries > kSlotSpinLimit) return false;
+        if (tries > 16) __nanosleep(tries > 4096 ? 256 : 32);
+        v = *p;
+    }
+    *p = kSlotEmpty;
+    return true;
+}
+
+__device__ __forceinline__ void norm_write(NormInfoDev *out, bool is_float, bool take_sqrt, bool ok, double fs,
+                                           unsigned long long is, unsigned long long nb, unsigned long long ne) {
+    if (!ok) {  // a slot never arrived: the result says so (lost_blocks can never be this large)
+        out->l2 = __longlong_as_double(0x7ff8000000000000ll);
+        out->l1 = 0;
+        out->lost_blocks = kSlotEmpty;
+        out->lost_elems = 0;
+        return;
+    }
+    out->l2 = is_float ? (take_sqrt ? sqrt(fs) : fs) : 0.0;  // l2 norms sum squares; l1 / weighted-l1 norms sum as they are
+    out->l1 = is_float ? 0ull : is;
+    out->lost_blocks = nb;
+    out->lost_elems = ne;
+}
+
+// Called by every thread of every CTA of a recovery / norm pass with the thread's own share (fs for float data,
+// is for integer data, lost blocks, lost elements).  The CTA's total goes to its slot with three plain stores,
+// and the CTA is done: nothing in the streaming part of the pass waits for the memory system on behalf of
+// the reduction.  The last CTAs of the grid (the watchers: one per 1024 CTAs) do the adding: watcher t collects
+// the slots of its contiguous share of the CTAs, thread i taking slots i, i + 256, ... in that order, then the
+// fixed tree of cta_sum; the last CTA collects the watchers' totals the same way and writes the result.
+// A watcher only ever waits for CTAs with a lower index than its own, which were dispatched before it and wait
+// for nobody, and every wait is bounded.  The order of every addition depends only on the grid size, so the
+// result is the same bits on every run.  This replaces a second launch: the pass and its reduction are one kernel.
 template <typename T>
-__global__ void __launch_bounds__(kThreads)
-k_reduce_partials(const typename Elem<T>::score_t *__restrict__ part, Geom g, LostSet S, double *tile_sum,
-                  unsigned long long *tile_l1, unsigned long long *tile_blocks, unsigned long long *tile_elems,
-                  unsigned *ticket, NormInfoDev *out, bool take_sqrt) {
+__device__ __forceinline__ void norm_epilogue(double fs, unsigned long long is, unsigned long long nb,
+                                              unsigned long long ne, const NormScratch &rs, NormInfoDev *out,
+                                              bool take_sqrt) {
+    typedef unsigned long long u64;
+    constexpr bool kF = std::is_same<T, float>::value;
     __shared__ double shd[kThreads / 32];
-    __shared__ unsigned long long shu[kThreads / 32];
-    __shared__ bool is_last;
-    griddep_wait();
-    const uint64_t base = (uint64_t)blockIdx.x * kReduceTile;
-    double fs = 0.0;
-    unsigned long long is = 0, nb = 0, ne = 0;
-    uint32_t bj[kReducePer];
-    bool ok[kReducePer];
-#pragma unroll
-    for (int j = 0; j < kReducePer; ++j) ok[j] = S.block_of(base + threadIdx.x + (uint64_t)j * kThreads, bj[j]);
-    typename Elem<T>::score_t pj[kReducePer];
-#pragma unroll
-    for (int j = 0; j < kReducePer; ++j) pj[j] = ok[j] ? part[bj[j]] : (typename Elem<T>::score_t)0;
-#pragma unroll
-    for (int j = 0; j < kReducePer; ++j)
-        if (ok[j]) {
-            uint64_t beg, len;
-            g.range(bj[j], beg, len);
-            ++nb;
-            ne += len;
-            if (std::is_same<T, float>::value) fs += (double)pj[j];
-            else is += (unsigned long long)pj[j];
-        }
-    fs = cta_sum<double>(fs, shd);
-    is = cta_sum<unsigned long long>(is, shu);
-    nb = cta_sum<unsigned long long>(nb, shu);
-    ne = cta_sum<unsigned long long>(ne, shu);
+    __shared__ u64 shu[kThreads / 32];
+    if (kF) fs = cta_sum<double>(fs, shd);
+    else is = cta_sum<u64>(is, shu);
+    nb = cta_sum<u64>(nb, shu);
+    ne = cta_sum<u64>(ne, shu);
+    const unsigned grid = gridDim.x;
+    if (grid == 1) {
+        if (threadIdx.x == 0) norm_write(out, kF, take_sqrt, true, fs, is, nb, ne);
+        return;
+    }
     if (threadIdx.x == 0) {
-        tile_sum[blockIdx.x] = fs;
-        tile_l1[blockIdx.x] = is;
-        tile_blocks[blockIdx.x] = nb;
-        tile_elems[blockIdx.x] = ne;
-        __threadfence();
-        is_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+        u64 v = is;
+        if (kF) v = fs != fs ? 0x7ff8000000000000ull : (u64)__double_as_longlong(fs);  // never the empty pattern
+        *reinterpret_cast<volatile u64 *>(rs.cta_val + blockIdx.x) = v;
+        *reinterpret_cast<volatile u64 *>(rs.cta_blocks + blockIdx.x) = nb;
+        *reinterpret_cast<volatile u64 *>(rs.cta_elems + blockIdx.x) = ne;
+    }
+    const unsigned n_watch = norm_watchers(grid);
+    if (blockIdx.x < grid - n_watch) return;
+
+    // ---- watcher t: the slots of CTAs [lo, hi)
+    const unsigned t = blockIdx.x - (grid - n_watch);
+    const unsigned share = (grid + n_watch - 1) / n_watch;
+    const unsigned lo = t * share, hi = lo + share < grid ? lo + share : grid;
+    bool ok = true;
+    fs = 0.0, is = 0, nb = 0, ne = 0;
+    constexpr int kAhead = 4;  // slots per thread whose loads are in flight together
+    for (unsigned base = lo + threadIdx.x; base < hi; base += kAhead * kThreads) {
+        u64 v[kAhead], b[kAhead], e[kAhead];
+#pragma unroll
+        for (int j = 0; j < kAhead; ++j) {
+            const unsigned i = base + j * kThreads;
+            if (i < hi) {
+                v[j] = slot_peek(rs.cta_val + i);
+                b[j] = slot_peek(rs.cta_blocks + i);
+                e[j] = slot_peek(rs.cta_elems + i);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kAhead; ++j) {
+            const unsigned i = base + j * kThreads;
+            if (i < hi) {
+                ok = slot_take(rs.cta_val + i, v[j]) && ok;
+                ok = slot_take(rs.cta_blocks + i, b[j]) && ok;
+                ok = slot_take(rs.cta_elems + i, e[j]) && ok;
+                if (kF) fs += __longlong_as_double((long long)v[j]);
+                else is += v[j];
+                nb += b[j];
+                ne += e[j];
+            }
+        }
+    }
+    ok = __syncthreads_and(ok) != 0;
+    if (kF) fs = cta_sum<double>(fs, shd);
+    else is = cta_sum<u64>(is, shu);
+    nb = cta_sum<u64>(nb, shu);
+    ne = cta_sum<u64>(ne, shu);
+    if (n_watch == 1) {
+        if (threadIdx.x == 0) norm_write(out, kF, take_sqrt, ok, fs, is, nb, ne);
+        return;
+    }
+    if (threadIdx.x == 0) {
+        u64 v = is;
+        if (kF) v = fs != fs ? 0x7ff8000000000000ull : (u64)__double_as_longlong(fs);
+        *reinterpret_cast<volatile u64 *>(rs.tile_val + t) = v;
+        *reinterpret_cast<volatile u64 *>(rs.tile_blocks + t) = ok ? nb : kSlotEmpty - 1;  // passes a failure on
+        *reinterpret_cast<volatile u64 *>(rs.tile_elems + t) = ne;
+    }
+    if (blockIdx.x != grid - 1) return;
+
+    // ---- the last CTA: the watchers' totals, in watcher order
+    fs = 0.0, is = 0, nb = 0, ne = 0;
+    if (threadIdx.x < n_watch) {
+        u64 v = slot_peek(rs.tile_val + threadIdx.x), b = slot_peek(rs.tile_blocks + threadIdx.x),
+            e = slot_peek(rs.tile_elems + threadIdx.x);
+        ok = slot_take(rs.tile_val + threadIdx.x, v) && ok;
+        ok = slot_take(rs.tile_blocks + threadIdx.x, b) && ok;
+        ok = slot_take(rs.tile_elems + threadIdx.x, e) && ok;
+        if (b == kSlotEmpty - 1) ok = false, b = 0;
+        if (kF) fs = __longlong_as_double((long long)v);
+        else is = v;
+        nb = b;
+        ne = e;
+    }
+    ok = __syncthreads_and(ok) != 0;
+    if (kF) fs = cta_sum<double>(fs, shd);
+    else is = cta_sum<u64>(is, shu);
+    nb = cta_sum<u64>(nb, shu);
+    ne = cta_sum<u64>(ne, shu);
+    if (threadIdx.x == 0) norm_write(out, kF, take_sqrt, ok, fs, is, nb, ne);
+}
+
+// ---- a4 / a5: perturbation over the lost set, optional restore, and its norm: one launch -----------
+
+// Exclusive prefix sum of one value per thread over a CTA of NT threads; *total gets the sum.
+template <typename W, int NT = kThreads>
+__device__ __forceinline__ W cta_excl_scan(W v, W *sh /*NT/32*/, W *total) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    W inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        W n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
     }
     __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    fs = 0.0; is = 0; nb = 0; ne = 0;
-    for (unsigned t = threadIdx.x; t < gridDim.x; t += kThreads) {
-        fs += *reinterpret_cast<volatile double *>(tile_sum + t);
-        is += *reinterpret_cast<volatile unsigned long long *>(tile_l1 + t);
-        nb += *reinterpret_cast<volatile unsigned long long *>(tile_blocks + t);
-        ne += *reinterpret_cast<volatile unsigned long long *>(tile_elems + t);
+    if (lane == 31) sh[w] = inc;
+    __syncthreads();
+    W before = 0, all = 0;
+#pragma unroll
+    for (int i = 0; i < NT / 32; ++i) {
+        W t = sh[i];
+        if (i < w) before += t;
+        all += t;
     }
-    fs = cta_sum<double>(fs, shd);
-    is = cta_sum<unsigned long long>(is, shu);
-    nb = cta_sum<unsigned long long>(nb, shu);
-    ne = cta_sum<unsigned long long>(ne, shu);
-    if (threadIdx.x == 0) {
-        out->l2 = take_sqrt ? sqrt(fs) : fs;  // l2 norms sum squares; l1 / weighted-l1 norms sum as they are
-        out->l1 = is;
-        out->lost_blocks = nb;
-        out->lost_elems = ne;
-        *ticket = 0;
+    if (total) *total = all;
+    return before + inc - v;
+}
+
+// Launch shape of the pass: one group of lanes per lost block; a per-block mask is cut into chunks of `chunk`
+// mask entries (a multiple of kThreads), one CTA each.
+constexpr unsigned kMaxMaskChunk = 4 * kThreads;
+struct RecoverShape {
+    unsigned grid;
+    unsigned chunk;
+};
+inline RecoverShape recover_shape(int mode, uint64_t n_work, int group_lanes) {
+    RecoverShape r{1, (unsigned)kThreads};
+    uint64_t want;
+    if (mode == 2) {
+        r.chunk = group_lanes < 32 ? 2 * kThreads : kThreads;  // short blocks: more of them per CTA
+        want = (n_work + r.chunk - 1) / r.chunk;
+    } else {
+        const uint64_t groups = kThreads / group_lanes;
+        want = (n_work + groups - 1) / groups;
     }
+    r.grid = (unsigned)(want < 1 ? 1 : want);
+    return r;
+}
+// CTAs of the largest launch recover_shape can give for a layout of n_blocks blocks.
+inline uint64_t recover_max_ctas(uint64_t n_blocks, int group_lanes) {
+    return (n_blocks + kThreads / group_lanes - 1) / (kThreads / group_lanes) + 1;
+}
+
+// A block's partial enters the sum as the value a score would store (rounded to float32 for float data), so that
+// the squared perturbation of a lost set is exactly the sum of the scores of its blocks.
+template <typename T, int NORM, int G, bool VEC, bool WRITE>
+__global__ void __launch_bounds__(kThreads)
+k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S, unsigned chunk,
+                 const float *__restrict__ weight, NormScratch rs, NormInfoDev *out) {
+    using E = Elem<T, NORM>;
+    typedef unsigned long long u64;
+    constexpr int kGroups = kThreads / G;
+    constexpr bool kF = std::is_same<T, float>::value;
+    const int lane = threadIdx.x & (G - 1), gi = threadIdx.x / G;
+    double fs = 0.0;
+    u64 is = 0, nb = 0, ne = 0;
+    if (S.mode == 2) {
+        // Per-block mask: the CTA takes `chunk` consecutive mask entries, writes the ids of the lost blocks
+        // among them, in order, to a list in shared memory, and its groups walk that list side by side, so
+        // that every group has a lost block to work on however sparse the mask is.
+        __shared__ uint32_t sh_list[kMaxMaskChunk];
+        __shared__ unsigned sh_scan[kThreads / 32];
+        const unsigned per = chunk / kThreads;  // consecutive entries per thread, 1..4
+        const u64 first = (u64)blockIdx.x * chunk + (u64)threadIdx.x * per;
+        unsigned bits = 0;
+        for (unsigned j = 0; j < per; ++j)
+            if (first + j < g.n_blocks && S.mask[first + j] != 0) bits |= 1u << j;
+        unsigned total;
+        unsigned pos = cta_excl_scan<unsigned, kThreads>(__popc(bits), sh_scan, &total);
+        for (unsigned j = 0; j < per; ++j)
+            if (bits >> j & 1u) sh_list[pos++] = (uint32_t)(first + j);
+        __syncthreads();
+        for (unsigned i0 = 0; i0 < total; i0 += kGroups) {  // same trip count for every thread of the CTA
+            const unsigned i = i0 + gi;
+            const bool valid = i < total;
+            uint32_t b = 0;
+            uint64_t beg = 0, len = 0;
+            if (valid) {
+                b = sh_list[i];
+                g.range(b, beg, len);
+            }
+            const typename E::wide_t s = block_distance<T, NORM, G, VEC, WRITE>(x, z, beg, len, lane);
+            if (valid && lane == 0) {
+                const typename E::score_t sc = weighted<E>(s, weight, b);
+                if (kF) fs += (double)sc;
+                else is += (u64)sc;
+                ++nb;
+                ne += len;
+            }
+        }
+    } else {
+        const uint64_t w = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
+        uint32_t b = 0;
+        const bool valid = S.block_of(w, b);
+        uint64_t beg = 0, len = 0;
+        if (valid) g.range(b, beg, len);
+        const typename E::wide_t s = block_distance<T, NORM, G, VEC, WRITE>(x, z, beg, len, lane);
+        if (valid && lane == 0) {
+            const typename E::score_t sc = weighted<E>(s, weight, b);
+            if (kF) fs = (double)sc;
+            else is = (u64)sc;
+            nb = 1;
+            ne = len;
+        }
+    }
+    norm_epilogue<T>(fs, is, nb, ne, rs, out, NORM == kNormDefault);
+}
+
+// Lost shards as a per-block mask, for lost sets with more runs than LostSet holds.  Up to kShardsByValue shard
+// flags travel inside the launch parameters (so the call reads no host memory after it returns and can be
+// recorded by stream capture); longer masks are read from device memory.
+constexpr int kShardsByValue = 1024;
+struct ShardFlags {
+    uint8_t lost[kShardsByValue];
+};
+static __global__ void __launch_bounds__(kThreads)
+k_expand_shards(Geom g, ShardFlags by_value, const uint8_t *__restrict__ shard_mask, uint8_t *__restrict__ block_mask) {
+    const uint64_t b = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (b >= g.n_blocks) return;
+    const uint32_t s = g.shard_of((uint32_t)b);
+    block_mask[b] = (shard_mask ? shard_mask[s] : by_value.lost[s]) != 0;
+}
+
+// ---- reduction of per-block partials as a kernel of its own -----------------------
+// (layouts cut into segments: their per-block partials come from a combine kernel, see segments.cuh)
+
+constexpr int kReduceTile = 1024;  // work items per CTA in the reduction
+constexpr int kReducePer = kReduceTile / kThreads;
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+k_reduce_partials(const typename Elem<T>::score_t *__restrict__ part, Geom g, LostSet S, NormScratch rs,
+                  NormInfoDev *out, bool take_sqrt) {
+    double fs = 0.0;
+    unsigned long long is = 0, nb = 0, ne = 0;
+    const uint64_t base = (uint64_t)blockIdx.x * kReduceTile;
+#pragma unroll
+    for (int j = 0; j < kReducePer; ++j) {
+        uint32_t b;
+        if (S.block_of(base + threadIdx.x + (uint64_t)j * kThreads, b)) {
+            uint64_t beg, len;
+            g.range(b, beg, len);
+            ++nb;
+            ne += len;
+            if (std::is_same<T, float>::value) fs += (double)part[b];
+            else is += (unsigned long long)part[b];
+        }
+    }
+    norm_epilogue<T>(fs, is, nb, ne, rs, out, take_sqrt);
 }
 
 // ---- plain copy (z := x at init, checkpoint reload) -------------------------

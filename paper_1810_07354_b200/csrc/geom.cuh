@@ -42,6 +42,31 @@ struct Geom {
     }
 };
 
+// Lengths of consecutive blocks, without a division per block: the row position of the first block is worked
+// out once and then counted up.
+struct BlockLens {
+    const Geom &g;
+    uint32_t b, j;  // current block and its position within its row (implicit layouts)
+    __device__ __forceinline__ BlockLens(const Geom &geom, uint32_t first) : g(geom), b(first), j(0) {
+        if (!g.boff && g.blocks_per_row > 1) j = first % g.blocks_per_row;
+    }
+    // length of the current block; moves on to the next one
+    __device__ __forceinline__ uint64_t next() {
+        uint64_t len;
+        if (g.boff) {
+            len = g.boff[b + 1] - g.boff[b];
+        } else if (g.blocks_per_row == 1) {
+            len = g.row_len;
+        } else {
+            const uint64_t rem = g.row_len - (uint64_t)j * g.block_elems;
+            len = rem < g.block_elems ? rem : (uint64_t)g.block_elems;
+            if (++j == g.blocks_per_row) j = 0;
+        }
+        ++b;
+        return len;
+    }
+};
+
 // The lost set S of a recovery (Section 4.1), as a list of work items that the
 // recovery kernels map to blocks.
 //   mode 0: every block is lost; work item w is block w.

@@ -17,18 +17,24 @@ __device__ __forceinline__ void copy_block_2dst(const U *__restrict__ src, U *__
     U c[4], nx[4];
     uint64_t u = lane;
     bool have = u < n;
+    // Loads are unconditional (a unit past the end re-reads the block's last unit; it is never stored), so that the
+    // four of a batch are issued back to back instead of one per branch.
     if (have) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (u + (uint64_t)j * G < n) c[j] = ld_stream(src + u + (uint64_t)j * G);
+        for (int j = 0; j < 4; ++j) {
+            const uint64_t i = u + (uint64_t)j * G;
+            c[j] = ld_stream(src + (i < n ? i : n - 1));
+        }
     }
     while (have) {
         const uint64_t un = u + step;
         const bool more = un < n;
         if (more) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (un + (uint64_t)j * G < n) nx[j] = ld_stream(src + un + (uint64_t)j * G);
+            for (int j = 0; j < 4; ++j) {
+                const uint64_t i = un + (uint64_t)j * G;
+                nx[j] = ld_stream(src + (i < n ? i : n - 1));
+            }
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -49,12 +55,12 @@ template <int G, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 k_pack_update(const uint32_t *__restrict__ x, uint32_t *__restrict__ z, uint32_t *__restrict__ payload, Geom g,
               const uint32_t *__restrict__ sel, const unsigned long long *__restrict__ poff, unsigned long long k,
-              const unsigned long long *selected) {
+              const SaveInfoDev *info) {
     const int lane = threadIdx.x & (G - 1);
     const uint64_t j = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
     if (j >= k) return;
     griddep_wait();  // the selection that wrote sel / poff may still be running
-    if (j >= *selected) return;  // fewer blocks than asked for: only when the selection gave up (then 0)
+    if (info->error || j >= info->k) return;  // a selection that gave up selected nothing that may be copied
     uint64_t beg, len;
     g.range(sel[j], beg, len);
     const uint64_t dst = poff[j];

@@ -2,11 +2,13 @@
 // the extern "C" entry points declared in include/scar.h.  Every step of the
 // checkpoint / recovery pass runs in the kernels of block_pass.cuh, select.cuh
 // and pack.cuh; there is no CPU path.
+#include <algorithm>
 #include <cerrno>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <functional>
 #include <new>
 #include <type_traits>
 #include <vector>
@@ -61,27 +63,28 @@ struct scar_ctx {
     OutSet cur{};   // where the next save writes
     OutSet last{};  // what the most recent save wrote (views and result fetches read this)
     void *score = nullptr;  // float[B] or uint64[B]
-    void *part = nullptr;   // per-block perturbation partials, same type as score
+    void *part = nullptr;   // per-block perturbation partials, same type as score (segment mode only)
     uint64_t *d_boff = nullptr;
     // segment mode (layouts with very long blocks)
     bool seg_mode = false;
     Segs segs{};
     void *seg_part = nullptr;      // double[n_segs] or uint64[n_segs]
-    uint32_t *selpos = nullptr;    // B: position in the id list, 0xffffffff when not selected
     uint32_t *wide_blocks = nullptr;  // blocks with more than kWideSegs segments
     unsigned n_wide_blocks = 0;
     int norm = SCAR_NORM_DEFAULT;
     float *d_weight = nullptr;  // per-block weights of the norm, or nullptr
     float *d_weight_buf = nullptr;
-    uint8_t *d_shard_mask = nullptr;
+    uint8_t *d_shard_mask = nullptr;  // only for shard masks too long to travel in launch parameters
+    uint8_t *h_shard_mask = nullptr;  // pinned staging copy of such a mask
     uint8_t *d_block_mask = nullptr;  // only used when a shard mask has too many runs
     SelState *st = nullptr;
-    CtaArrays ca{};
     unsigned n_sel_tiles = 0;
     unsigned sel_grid = 1, sel_tiles_per_cta = 1;  // launch shape of the cooperative selection kernel
-    double *rt_sum = nullptr;
-    unsigned long long *rt_l1 = nullptr, *rt_blocks = nullptr, *rt_elems = nullptr;
-    unsigned n_red_tiles = 0;
+    bool arm_never = false;  // self-test: the next selection's waits expect an arrival that never comes
+    int n_sms = 1;
+    NormScratch rs{};  // per-CTA / per-tile partials and tickets of the fused norm reduction
+    unsigned long long *norm_scratch = nullptr;  // what rs points into
+    size_t norm_scratch_bytes = 0;
     NormInfoDev *d_norm = nullptr;
     SaveInfoDev *h_save = nullptr;  // pinned
     NormInfoDev *h_norm = nullptr;  // pinned
@@ -97,6 +100,7 @@ struct scar_ctx {
 
     // persistent copy of the running checkpoint (scar_ckpt_store_* / scar_ckpt_load_stored)
     std::vector<uint64_t> h_boff;  // host copy of explicit block offsets (empty for implicit layouts)
+    std::vector<uint64_t> longest_prefix;  // explicit layouts: [k] = elements of the k longest blocks
     char *io_stage = nullptr;      // pinned staging buffer for whole-checkpoint transfers
 
     std::vector<void *> owned;  // device allocations to free
@@ -232,14 +236,15 @@ void record(scar_ctx *c, int i) {
 }
 
 // a1
-template <typename T, int NORM> void launch_scores_as(scar_ctx *c) {
+// info: result record of the save this scoring pass belongs to (cleared by the kernel), or nullptr
+template <typename T, int NORM> void launch_scores_as(scar_ctx *c, SaveInfoDev *info) {
     using S = typename Elem<T, NORM>::score_t;
     dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
         constexpr int G = decltype(gl)::value;
         constexpr bool VEC = decltype(vec)::value;
         k_block_scores<T, NORM, G, VEC><<<grid_for_groups(c->g.n_blocks, G), kThreads, 0, c->stream>>>(
             static_cast<const T *>(c->x), static_cast<const T *>(c->z), c->g, c->d_weight, static_cast<S *>(c->score),
-            &c->st->key_or, c->st->hist[0], kHistBins);
+            c->st, info);
     });
     ++c->launches;
 }
@@ -249,18 +254,19 @@ unsigned grid_for_warps(uint64_t n_warps) { return (unsigned)((n_warps + kThread
 // Segment sums -> block totals: one warp per block, plus one CTA per block that has very many segments.
 template <typename T, int NORM>
 void launch_combine(scar_ctx *c, const typename Elem<T, NORM>::wide_t *sp, const uint8_t *mask,
-                    typename Elem<T, NORM>::score_t *out, unsigned long long *key_or, unsigned *hist0, int hist0_len) {
+                    typename Elem<T, NORM>::score_t *out, unsigned long long *key_or, SelState *sel_state,
+                    SaveInfoDev *info) {
     k_combine_segments<T, NORM, false><<<grid_for_warps(c->g.n_blocks), kThreads, 0, c->stream>>>(
-        c->segs, c->g.n_blocks, nullptr, sp, c->d_weight, mask, out, key_or, hist0, hist0_len);
+        c->segs, c->g.n_blocks, nullptr, sp, c->d_weight, mask, out, key_or, sel_state, info);
     ++c->launches;
     if (c->n_wide_blocks) {
         k_combine_segments<T, NORM, true><<<c->n_wide_blocks, kThreads, 0, c->stream>>>(
-            c->segs, c->g.n_blocks, c->wide_blocks, sp, c->d_weight, mask, out, key_or, nullptr, 0);
+            c->segs, c->g.n_blocks, c->wide_blocks, sp, c->d_weight, mask, out, key_or, nullptr, nullptr);
         ++c->launches;
     }
 }
 
-template <typename T, int NORM> void launch_segment_scores(scar_ctx *c) {
+template <typename T, int NORM> void launch_segment_scores(scar_ctx *c, SaveInfoDev *info) {
     using W = typename Elem<T, NORM>::wide_t;
     using S = typename Elem<T, NORM>::score_t;
     T *x = static_cast<T *>(c->x);
@@ -272,21 +278,21 @@ template <typename T, int NORM> void launch_segment_scores(scar_ctx *c) {
     else
         k_segment_pass<T, NORM, false, false><<<grid_for_warps(c->segs.n), kThreads, 0, c->stream>>>(x, z, c->g, c->segs,
                                                                                                   nullptr, sp);
-    launch_combine<T, NORM>(c, sp, nullptr, static_cast<S *>(c->score), &c->st->key_or, c->st->hist[0], kHistBins);
+    launch_combine<T, NORM>(c, sp, nullptr, static_cast<S *>(c->score), &c->st->key_or, c->st, info);
     ++c->launches;
 }
 
-void launch_scores(scar_ctx *c) {
+void launch_scores(scar_ctx *c, SaveInfoDev *info) {
     if (c->g.n_blocks == 0) return;
     if (c->seg_mode) {
-        if (c->dt == SCAR_I32) launch_segment_scores<int, kNormDefault>(c);
-        else if (c->norm == SCAR_NORM_L1) launch_segment_scores<float, kNormL1>(c);
-        else launch_segment_scores<float, kNormDefault>(c);
+        if (c->dt == SCAR_I32) launch_segment_scores<int, kNormDefault>(c, info);
+        else if (c->norm == SCAR_NORM_L1) launch_segment_scores<float, kNormL1>(c, info);
+        else launch_segment_scores<float, kNormDefault>(c, info);
         return;
     }
-    if (c->dt == SCAR_I32) launch_scores_as<int, kNormDefault>(c);
-    else if (c->norm == SCAR_NORM_L1) launch_scores_as<float, kNormL1>(c);
-    else launch_scores_as<float, kNormDefault>(c);
+    if (c->dt == SCAR_I32) launch_scores_as<int, kNormDefault>(c, info);
+    else if (c->norm == SCAR_NORM_L1) launch_scores_as<float, kNormL1>(c, info);
+    else launch_scores_as<float, kNormDefault>(c, info);
 }
 
 // a1 + a3 fused for k == B
@@ -302,52 +308,96 @@ template <typename T, int NORM> void launch_full_save(scar_ctx *c) {
     ++c->launches;
 }
 
-// a2: one cooperative launch (all CTAs resident, so its grid-wide barriers cannot deadlock)
-template <typename S> int launch_select(scar_ctx *c, const S *score, uint64_t k) {
+// a2: one cooperative launch (all CTAs resident, so its waits cannot deadlock).  The selection state must be
+// zero when the kernel starts: the scoring pass that precedes a prioritized save clears it (pre_cleared), any
+// other caller gets a memset here.
+template <typename S> int launch_select(scar_ctx *c, const S *score, uint64_t k, bool pre_cleared) {
+    if (!pre_cleared) {
+        CU_TRY(cudaMemsetAsync(reinterpret_cast<char *>(c->st) + kSelZeroFrom, 0, sizeof(SelState) - kSelZeroFrom,
+                               c->stream));
+        CU_TRY(cudaMemsetAsync(c->cur.info, 0, sizeof(SaveInfoDev), c->stream));
+    }
     unsigned long long kk = k;
-    unsigned nt = c->n_sel_tiles, per = c->sel_tiles_per_cta;
-    void *args[] = {&score, &c->g, &kk, &c->st, &c->ca, &c->cur.info, &c->cur.sel, &c->cur.poff, &nt, &per};
-    CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select<S>), dim3(c->sel_grid),
-                                       dim3(kThreads), args, 0, c->stream));
+    unsigned k32 = (unsigned)k, nt = c->n_sel_tiles, per = c->sel_tiles_per_cta, never = c->arm_never ? 1u : 0u;
+    c->arm_never = false;
+    if (per == 1) {  // the usual case: one tile per CTA
+        void *args[] = {&score, &c->g, &k32, &c->st, &c->cur.info, &c->cur.sel, &c->cur.poff, &never};
+        CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select_tile<S>), dim3(c->sel_grid),
+                                           dim3(kSelThreads), args, 0, c->stream));
+    } else {
+        void *args[] = {&score, &c->g, &kk, &c->st, &c->cur.info, &c->cur.sel, &c->cur.poff, &nt, &per, &never};
+        CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select<S, false>), dim3(c->sel_grid),
+                                           dim3(kSelThreads), args, 0, c->stream));
+    }
     ++c->launches;
     return SCAR_OK;
 }
 
-// Grid of the selection kernel: contiguous tile ranges over at most two CTAs per
-// SM (few enough that a barrier costs about a microsecond, and always resident).
+// Grid of the selection kernel: contiguous tile ranges over at most one CTA per SM (few enough that a meeting
+// of all CTAs costs a couple of microseconds, always resident, and fewer than the exchange has threads).
+template <typename S> int select_occupancy(int &occ) {
+    int o = 0;
+    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, k_select<S, false>, kSelThreads, 0));
+    occ = o < occ ? o : occ;
+    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, k_select_tile<S>, kSelThreads, 0));
+    occ = o < occ ? o : occ;
+    return SCAR_OK;
+}
+
 int plan_select(scar_ctx *c) {
-    int coop = 0, sms = 0, occ = 0, o = 0;
+    int coop = 0, sms = 0, occ = 1 << 30, rc;
     CU_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
     CU_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device));
-    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_select<float>, kThreads, 0));
-    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, k_select<unsigned long long>, kThreads, 0));
-    occ = o < occ ? o : occ;
-    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, k_select<unsigned>, kThreads, 0));
-    occ = o < occ ? o : occ;
+    if ((rc = select_occupancy<float>(occ)) != SCAR_OK || (rc = select_occupancy<unsigned long long>(occ)) != SCAR_OK ||
+        (rc = select_occupancy<unsigned>(occ)) != SCAR_OK)
+        return rc;
     if (!coop || sms < 1 || occ < 1) return SCAR_ERR_CUDA;
-    const unsigned cap = (unsigned)sms * (unsigned)(occ < 2 ? occ : 2);
+    c->n_sms = sms;
+    const unsigned cap = (unsigned)sms < (unsigned)kMaxSelCtas - 1 ? (unsigned)sms : (unsigned)kMaxSelCtas - 1;
     const unsigned nt = c->n_sel_tiles;
     c->sel_tiles_per_cta = (nt + cap - 1) / cap;
     c->sel_grid = (nt + c->sel_tiles_per_cta - 1) / c->sel_tiles_per_cta;
     return SCAR_OK;
 }
 
+// a1 + a3 fused for k == B on a segmented layout
+template <typename T, int NORM> void launch_full_save_segments_as(scar_ctx *c) {
+    using W = typename Elem<T, NORM>::wide_t;
+    using S = typename Elem<T, NORM>::score_t;
+    const T *x = static_cast<const T *>(c->x);
+    T *z = static_cast<T *>(c->z), *pay = static_cast<T *>(c->cur.payload);
+    W *sp = static_cast<W *>(c->seg_part);
+    const unsigned grid = grid_for_warps(c->segs.n);
+    if (c->g.vec_ok) k_segment_full_save<T, NORM, true><<<grid, kThreads, 0, c->stream>>>(x, z, pay, c->g, c->segs, sp);
+    else k_segment_full_save<T, NORM, false><<<grid, kThreads, 0, c->stream>>>(x, z, pay, c->g, c->segs, sp);
+    ++c->launches;
+    launch_combine<T, NORM>(c, sp, nullptr, static_cast<S *>(c->score), nullptr, nullptr, nullptr);
+    k_full_save_ids<S><<<(unsigned)((c->g.n_blocks + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(
+        c->g, static_cast<const S *>(c->score), c->cur.sel, c->cur.poff, c->cur.info);
+    ++c->launches;
+}
+
+void launch_full_save_segments(scar_ctx *c) {
+    if (c->dt == SCAR_I32) launch_full_save_segments_as<int, kNormDefault>(c);
+    else if (c->norm == SCAR_NORM_L1) launch_full_save_segments_as<float, kNormL1>(c);
+    else launch_full_save_segments_as<float, kNormDefault>(c);
+}
+
 // a3
 void launch_pack(scar_ctx *c, uint64_t k) {
     if (k == 0) return;
     if (c->seg_mode) {
-        cudaMemsetAsync(c->selpos, 0xff, c->g.n_blocks * 4, c->stream);
-        k_mark_selected<<<(unsigned)((k + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(c->cur.sel, c->cur.info,
-                                                                                              c->selpos);
         const uint32_t *x = static_cast<const uint32_t *>(c->x);
         uint32_t *z = static_cast<uint32_t *>(c->z), *pay = static_cast<uint32_t *>(c->cur.payload);
+        const unsigned want = grid_for_warps(c->segs.n), cap = (unsigned)c->n_sms * 8u;
+        const unsigned grid = want < cap ? want : cap;
         if (c->g.vec_ok)
-            k_pack_segments<true><<<grid_for_warps(c->segs.n), kThreads, 0, c->stream>>>(x, z, pay, c->g, c->segs,
-                                                                                       c->selpos, c->cur.poff);
+            launch_after(c, k_pack_segments<true>, grid, x, z, pay, c->g, c->segs, (const uint32_t *)c->cur.sel,
+                         (const unsigned long long *)c->cur.poff, (const SaveInfoDev *)c->cur.info);
         else
-            k_pack_segments<false><<<grid_for_warps(c->segs.n), kThreads, 0, c->stream>>>(x, z, pay, c->g, c->segs,
-                                                                                        c->selpos, c->cur.poff);
-        c->launches += 2;
+            launch_after(c, k_pack_segments<false>, grid, x, z, pay, c->g, c->segs, (const uint32_t *)c->cur.sel,
+                         (const unsigned long long *)c->cur.poff, (const SaveInfoDev *)c->cur.info);
+        ++c->launches;
         return;
     }
     dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
@@ -355,15 +405,21 @@ void launch_pack(scar_ctx *c, uint64_t k) {
         constexpr bool VEC = decltype(vec)::value;
         launch_after(c, k_pack_update<G, VEC>, grid_for_groups(k, G), static_cast<const uint32_t *>(c->x),
                      static_cast<uint32_t *>(c->z), static_cast<uint32_t *>(c->cur.payload), c->g, c->cur.sel,
-                     c->cur.poff, (unsigned long long)k, &c->cur.info->k);
+                     c->cur.poff, (unsigned long long)k, c->cur.info);
     });
     ++c->launches;
 }
 
-// a4 / a5
-template <typename T, int NORM> void launch_recover_as(scar_ctx *c, const LostSet &S, bool write) {
+// a4 / a5: one launch; the kernel's last CTA finishes the norm
+template <typename T, int NORM> int launch_recover_as(scar_ctx *c, const LostSet &S, bool write) {
     using Sc = typename Elem<T, NORM>::score_t;
-    if (c->seg_mode && S.n_work > 0) {
+    if (S.n_work == 0) {  // nothing lost: zero perturbation, x untouched
+        CU_TRY(cudaMemsetAsync(c->d_norm, 0, sizeof(NormInfoDev), c->stream));
+        record(c, 4);
+        record(c, 5);
+        return SCAR_OK;
+    }
+    if (c->seg_mode) {
         // S is "all blocks" (mode 0) or a per-block mask (mode 2) here: enqueue_recover turns shard runs into a mask
         using W = typename Elem<T, NORM>::wide_t;
         T *x = static_cast<T *>(c->x);
@@ -379,44 +435,42 @@ template <typename T, int NORM> void launch_recover_as(scar_ctx *c, const LostSe
             else k_segment_pass<T, NORM, false, false><<<grid, kThreads, 0, c->stream>>>(x, z, c->g, c->segs, mask, sp);
         }
         ++c->launches;
-        launch_combine<T, NORM>(c, sp, mask, static_cast<Sc *>(c->part), nullptr, nullptr, 0);
-    } else if (S.n_work > 0) {
-        dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
-            constexpr int G = decltype(gl)::value;
-            constexpr bool VEC = decltype(vec)::value;
-            // a per-block mask with several blocks per warp is walked 32 blocks per warp
-            const unsigned grid = (G < 32 && S.mode == 2) ? (unsigned)((S.n_work + kThreads - 1) / kThreads)
-                                                          : grid_for_groups(S.n_work, G);
-            if (write)
-                k_recover_blocks<T, NORM, G, VEC, true><<<grid, kThreads, 0, c->stream>>>(
-                    static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, c->d_weight,
-                    static_cast<Sc *>(c->part));
-            else
-                k_recover_blocks<T, NORM, G, VEC, false><<<grid, kThreads, 0, c->stream>>>(
-                    static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, c->d_weight,
-                    static_cast<Sc *>(c->part));
-        });
+        launch_combine<T, NORM>(c, sp, mask, static_cast<Sc *>(c->part), nullptr, nullptr, nullptr);
+        record(c, 4);
+        const uint64_t tiles = (S.n_work + kReduceTile - 1) / kReduceTile;
+        k_reduce_partials<T><<<(unsigned)tiles, kThreads, 0, c->stream>>>(static_cast<const Sc *>(c->part), c->g, S,
+                                                                         c->rs, c->d_norm, NORM == kNormDefault);
         ++c->launches;
+        record(c, 5);
+        return SCAR_OK;
     }
-    record(c, 4);
-    uint64_t tiles = (S.n_work + kReduceTile - 1) / kReduceTile;
-    if (tiles == 0) tiles = 1;
-    launch_after(c, k_reduce_partials<T>, (unsigned)tiles, static_cast<const Sc *>(c->part), c->g, S, c->rt_sum,
-                 c->rt_l1, c->rt_blocks, c->rt_elems, &c->st->ticket_reduce, c->d_norm, NORM == kNormDefault);
+    const RecoverShape sh = recover_shape(S.mode, S.n_work, c->group_lanes);
+    dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
+        constexpr int G = decltype(gl)::value;
+        constexpr bool VEC = decltype(vec)::value;
+        if (write)
+            k_recover_blocks<T, NORM, G, VEC, true><<<sh.grid, kThreads, 0, c->stream>>>(
+                static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, sh.chunk, c->d_weight, c->rs, c->d_norm);
+        else
+            k_recover_blocks<T, NORM, G, VEC, false><<<sh.grid, kThreads, 0, c->stream>>>(
+                static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, sh.chunk, c->d_weight, c->rs, c->d_norm);
+    });
     ++c->launches;
+    record(c, 4);
     record(c, 5);
+    return SCAR_OK;
 }
 
-void launch_recover(scar_ctx *c, const LostSet &S, bool write) {
-    if (c->dt == SCAR_I32) launch_recover_as<int, kNormDefault>(c, S, write);
-    else if (c->norm == SCAR_NORM_L1) launch_recover_as<float, kNormL1>(c, S, write);
-    else launch_recover_as<float, kNormDefault>(c, S, write);
+int launch_recover(scar_ctx *c, const LostSet &S, bool write) {
+    if (c->dt == SCAR_I32) return launch_recover_as<int, kNormDefault>(c, S, write);
+    if (c->norm == SCAR_NORM_L1) return launch_recover_as<float, kNormL1>(c, S, write);
+    return launch_recover_as<float, kNormDefault>(c, S, write);
 }
 
 int copy_elems(scar_ctx *c, void *dst, const void *src, uint64_t n) {
     if (n == 0) return SCAR_OK;
-    uint64_t want = ((n >> 2) + kThreads - 1) / kThreads;
-    unsigned grid = (unsigned)(want < 1 ? 1 : (want > 148u * 16u ? 148u * 16u : want));
+    const uint64_t want = ((n >> 2) + kThreads - 1) / kThreads, cap = (uint64_t)c->n_sms * 16u;
+    unsigned grid = (unsigned)(want < 1 ? 1 : (want > cap ? cap : want));
     k_copy_elems<<<grid, kThreads, 0, c->stream>>>(static_cast<uint32_t *>(dst), static_cast<const uint32_t *>(src), n);
     ++c->launches;
     CU_TRY(cudaGetLastError());
@@ -441,6 +495,12 @@ int fetch_save(scar_ctx *c, scar_save_info *out) {
 int fetch_norm(scar_ctx *c, scar_norm_info *out) {
     CU_TRY(cudaMemcpyAsync(c->h_norm, c->d_norm, sizeof(NormInfoDev), cudaMemcpyDeviceToHost, c->stream));
     CU_TRY(cudaStreamSynchronize(c->stream));
+    if (c->h_norm->lost_blocks == kSlotEmpty) {
+        // A bounded wait of the reduction gave up (a slot never arrived).  Slots may be left in any state:
+        // empty them all before the next pass.
+        CU_TRY(cudaMemsetAsync(c->norm_scratch, 0xff, c->norm_scratch_bytes, c->stream));
+        return SCAR_ERR_TIMEOUT;
+    }
     out->l2 = c->h_norm->l2;
     out->l1 = c->h_norm->l1;
     out->lost_blocks = c->h_norm->lost_blocks;
@@ -458,66 +518,88 @@ int k_from_r(double r, uint64_t n_blocks, uint64_t *k) {
     return SCAR_OK;
 }
 
-// Common start of every save: in drain mode the save must fit the slot it writes to.
-int begin_save(scar_ctx *c, uint64_t k) {
+// Most elements any k blocks of the layout can hold (the k longest blocks).
+uint64_t save_bound(const scar_ctx *c, uint64_t k) {
+    if (!c->longest_prefix.empty()) return c->longest_prefix[k];
+    if (c->g.n_blocks == 0) return 0;
+    const uint64_t per_row = c->g.blocks_per_row, blk = c->g.row_len < c->g.block_elems ? c->g.row_len : c->g.block_elems;
+    const uint64_t tail = c->g.row_len - (per_row - 1) * c->g.block_elems;  // last block of a row, <= blk
+    const uint64_t n_full = tail < blk ? (c->g.n_blocks / per_row) * (per_row - 1) : c->g.n_blocks;
+    return (k < n_full ? k : n_full) * blk + (k > n_full ? (k - n_full) * tail : 0);
+}
+
+// Before anything is enqueued: in drain mode the save must fit the slot it writes to.  Changes nothing.
+int save_fits(const scar_ctx *c, uint64_t k) {
+    if (!c->drain) return SCAR_OK;
+    const DrainSlot &sl = c->slot[c->cur_slot];
+    if (sl.state >= 2) return SCAR_ERR_STATE;  // both slots are still out: release the older ticket first
+    if (k > c->drain_cap_k || save_bound(c, k) > c->drain_cap_elems) return SCAR_ERR_CAPACITY;
+    return SCAR_OK;
+}
+
+// After every launch of a save went through: only now does the context point at the new save.
+void commit_save(scar_ctx *c, uint64_t k) {
     if (c->drain) {
         DrainSlot &sl = c->slot[c->cur_slot];
-        if (sl.state >= 2) return SCAR_ERR_STATE;  // both slots are still out: release the older ticket first
-        if (k > c->drain_cap_k || k * c->max_block_len > c->drain_cap_elems) return SCAR_ERR_CAPACITY;
         sl.k = k;
         sl.state = 1;
     }
     c->last = c->cur;
-    return SCAR_OK;
+    c->have_save = true;
 }
 
 int enqueue_save(scar_ctx *c, uint64_t k) {
-    const int rc_begin = begin_save(c, k);
-    if (rc_begin != SCAR_OK) return rc_begin;
+    const int rc_fit = save_fits(c, k);
+    if (rc_fit != SCAR_OK) return rc_fit;
     c->last_call = 1;
     c->ran_select = c->ran_pack = false;
     record(c, 0);
     if (c->g.n_blocks == 0) {
         CU_TRY(cudaMemsetAsync(c->cur.info, 0, sizeof(SaveInfoDev), c->stream));
         CU_TRY(cudaMemsetAsync(c->cur.poff, 0, sizeof(unsigned long long), c->stream));
-        c->have_save = true;
+        commit_save(c, k);
         return SCAR_OK;
     }
-    if (k == c->g.n_blocks && !c->seg_mode) {
+    if (k == c->g.n_blocks) {
         // Full checkpoint: nothing to choose, so one fused pass scores, packs and refreshes z.
         CU_TRY(cudaMemsetAsync(c->cur.info, 0, sizeof(SaveInfoDev), c->stream));
-        if (c->dt == SCAR_I32) launch_full_save<int, kNormDefault>(c);
+        if (c->seg_mode) launch_full_save_segments(c);
+        else if (c->dt == SCAR_I32) launch_full_save<int, kNormDefault>(c);
         else if (c->norm == SCAR_NORM_L1) launch_full_save<float, kNormL1>(c);
         else launch_full_save<float, kNormDefault>(c);
         record(c, 1);
         record(c, 2);
         record(c, 3);
-        c->ran_select = c->ran_pack = true;
         CU_TRY(cudaGetLastError());
-        c->have_save = true;
+        c->ran_select = c->ran_pack = true;
+        commit_save(c, k);
         return SCAR_OK;
     }
-    launch_scores(c);
+    launch_scores(c, c->cur.info);
     record(c, 1);
-    const int rc_sel = c->dt == SCAR_F32
-                           ? launch_select<float>(c, static_cast<const float *>(c->score), k)
-                           : launch_select<unsigned long long>(c, static_cast<const unsigned long long *>(c->score), k);
-    if (rc_sel != SCAR_OK) return rc_sel;
-    c->ran_select = true;
+    const int rc_sel =
+        c->dt == SCAR_F32
+            ? launch_select<float>(c, static_cast<const float *>(c->score), k, true)
+            : launch_select<unsigned long long>(c, static_cast<const unsigned long long *>(c->score), k, true);
+    if (rc_sel != SCAR_OK) {
+        cudaGetLastError();
+        return rc_sel;
+    }
     record(c, 2);
     launch_pack(c, k);
-    c->ran_pack = k > 0;
     record(c, 3);
     CU_TRY(cudaGetLastError());
-    c->have_save = true;
+    c->ran_select = true;
+    c->ran_pack = k > 0;
+    commit_save(c, k);
     return SCAR_OK;
 }
 
 // Saves with a selector that does not look at distances (Section 5.4: `round`, `random`):
 // no scoring pass; selection, then the same pack + cache refresh as a prioritized save.
 int enqueue_baseline_save(scar_ctx *c, uint64_t k, const uint32_t *d_priorities) {
-    const int rc_begin = begin_save(c, k);
-    if (rc_begin != SCAR_OK) return rc_begin;
+    const int rc_fit = save_fits(c, k);
+    if (rc_fit != SCAR_OK) return rc_fit;
     c->last_call = 1;
     c->ran_select = c->ran_pack = false;
     record(c, 0);
@@ -525,26 +607,29 @@ int enqueue_baseline_save(scar_ctx *c, uint64_t k, const uint32_t *d_priorities)
     if (c->g.n_blocks == 0) {
         CU_TRY(cudaMemsetAsync(c->cur.info, 0, sizeof(SaveInfoDev), c->stream));
         CU_TRY(cudaMemsetAsync(c->cur.poff, 0, sizeof(unsigned long long), c->stream));
-        c->have_save = true;
+        commit_save(c, k);
         return SCAR_OK;
     }
     if (d_priorities) {
-        const int rc = launch_select<unsigned>(c, d_priorities, k);
-        if (rc != SCAR_OK) return rc;
+        const int rc = launch_select<unsigned>(c, d_priorities, k, false);
+        if (rc != SCAR_OK) {
+            cudaGetLastError();
+            return rc;
+        }
     } else {
         const unsigned grid = (unsigned)((k + kThreads - 1) / kThreads);
         k_select_round<<<grid ? grid : 1, kThreads, 0, c->stream>>>(c->g, c->round_cursor, k, c->cur.sel, c->cur.poff,
                                                                       c->cur.info);
         ++c->launches;
-        c->round_cursor = (c->round_cursor + k) % c->g.n_blocks;
     }
-    c->ran_select = true;
     record(c, 2);
     launch_pack(c, k);
-    c->ran_pack = k > 0;
     record(c, 3);
     CU_TRY(cudaGetLastError());
-    c->have_save = true;
+    if (!d_priorities) c->round_cursor = (c->round_cursor + k) % c->g.n_blocks;  // only once the save is on its way
+    c->ran_select = true;
+    c->ran_pack = k > 0;
+    commit_save(c, k);
     return SCAR_OK;
 }
 
@@ -556,10 +641,23 @@ int enqueue_recover(scar_ctx *c, const LostSet &S, bool write) {
         c->have_norm = true;
         return SCAR_OK;
     }
-    launch_recover(c, S, write);
+    const int rc = launch_recover(c, S, write);
+    if (rc != SCAR_OK) return rc;
     CU_TRY(cudaGetLastError());
     c->have_norm = true;
     return SCAR_OK;
+}
+
+// Element range of block b from the host copy of the layout.
+void host_range(const scar_ctx *c, uint64_t b, uint64_t &beg, uint64_t &len) {
+    if (!c->h_boff.empty()) {
+        beg = c->h_boff[b];
+        len = c->h_boff[b + 1] - beg;
+        return;
+    }
+    const uint64_t row = b / c->g.blocks_per_row, j = b % c->g.blocks_per_row, o = j * c->g.block_elems;
+    beg = row * c->g.row_len + o;
+    len = c->g.row_len - o < c->g.block_elems ? c->g.row_len - o : c->g.block_elems;
 }
 
 LostSet all_lost(const scar_ctx *c) {
@@ -579,7 +677,10 @@ LostSet block_mask_set(const scar_ctx *c, const uint8_t *d_lost_blocks) {
 
 // Lost shards -> runs of consecutive lost blocks (adjacent lost shards merge,
 // shards that own no block vanish).  With more runs than LostSet can carry,
-// the shard mask is expanded into a per-block mask on the device instead.
+// the shard mask is expanded into a per-block mask on the device instead: up
+// to kShardsByValue shard flags travel in the launch parameters, longer masks
+// go through a pinned buffer of the context (so no copy ever reads the
+// caller's array after this returns).
 int shard_set(scar_ctx *c, const uint8_t *h_lost_shards, LostSet &S) {
     const uint64_t B = c->g.n_blocks, n_sh = c->g.n_shards;
     S = LostSet{};
@@ -606,9 +707,19 @@ int shard_set(scar_ctx *c, const uint8_t *h_lost_shards, LostSet &S) {
         S.run_start[S.n_runs] = (uint32_t)work;
     }
     S.n_work = work;
-    if (!overflow && !c->seg_mode) return SCAR_OK;  // segment mode walks segments, so it always wants a block mask
-    CU_TRY(cudaMemcpyAsync(c->d_shard_mask, h_lost_shards, n_sh, cudaMemcpyHostToDevice, c->stream));
-    k_expand_shards<<<(unsigned)((B + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(c->g, c->d_shard_mask,
+    if (B == 0 || (!overflow && !c->seg_mode)) return SCAR_OK;  // segment mode walks segments: it always wants a block mask
+    ShardFlags flags{};
+    const uint8_t *d_mask = nullptr;
+    if (n_sh <= (uint64_t)kShardsByValue) {
+        memcpy(flags.lost, h_lost_shards, n_sh);
+    } else {
+        // the pinned buffer may still be the source of an earlier call's copy
+        CU_TRY(cudaStreamSynchronize(c->stream));
+        memcpy(c->h_shard_mask, h_lost_shards, n_sh);
+        CU_TRY(cudaMemcpyAsync(c->d_shard_mask, c->h_shard_mask, n_sh, cudaMemcpyHostToDevice, c->stream));
+        d_mask = c->d_shard_mask;
+    }
+    k_expand_shards<<<(unsigned)((B + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(c->g, flags, d_mask,
                                                                                           c->d_block_mask);
     ++c->launches;
     CU_TRY(cudaGetLastError());
@@ -662,10 +773,12 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     c->group_lanes = pick_group_lanes(g);
     if (layout->block_offsets) {
         c->h_boff.assign(layout->block_offsets, layout->block_offsets + g.n_blocks + 1);
-        for (uint64_t b = 0; b < g.n_blocks; ++b) {
-            const uint64_t len = layout->block_offsets[b + 1] - layout->block_offsets[b];
-            if (len > c->max_block_len) c->max_block_len = len;
-        }
+        std::vector<uint64_t> lens(g.n_blocks);
+        for (uint64_t b = 0; b < g.n_blocks; ++b) lens[b] = layout->block_offsets[b + 1] - layout->block_offsets[b];
+        std::sort(lens.begin(), lens.end(), std::greater<uint64_t>());
+        c->longest_prefix.assign(g.n_blocks + 1, 0);
+        for (uint64_t b = 0; b < g.n_blocks; ++b) c->longest_prefix[b + 1] = c->longest_prefix[b] + lens[b];
+        c->max_block_len = g.n_blocks ? lens[0] : 0;
     } else {
         c->max_block_len = g.row_len < g.block_elems ? g.row_len : g.block_elems;
     }
@@ -674,9 +787,7 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     const size_t score_bytes = (dt == SCAR_F32 ? 4 : 8) * B;
     c->n_sel_tiles = (unsigned)((B + kSelTile - 1) / kSelTile);
     if (c->n_sel_tiles == 0) c->n_sel_tiles = 1;
-    c->n_red_tiles = (unsigned)((B + kReduceTile - 1) / kReduceTile);
-    if (c->n_red_tiles == 0) c->n_red_tiles = 1;
-    const unsigned nr = c->n_red_tiles;
+    const bool long_blocks = c->max_block_len > 2 * kSegElems;
 
     rc = SCAR_OK;
     auto A = [&](auto **p, size_t bytes) {
@@ -685,24 +796,30 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     A(&c->z, N * 4);
     A(&c->cur.payload, N * 4);
     A(&c->score, score_bytes);
-    A(&c->part, score_bytes);
+    if (long_blocks) A(&c->part, score_bytes);
     A(&c->cur.sel, B * 4);
     A(&c->cur.poff, (B + 1) * 8);
-    A(&c->d_shard_mask, g.n_shards);
+    if (g.n_shards > (uint32_t)kShardsByValue) {
+        A(&c->d_shard_mask, g.n_shards);
+        if (rc == SCAR_OK) {
+            void *q = nullptr;
+            if (cudaMallocHost(&q, g.n_shards) != cudaSuccess) {
+                cudaGetLastError();
+                rc = SCAR_ERR_ALLOC;
+            } else {
+                c->owned_host.push_back(q);
+                c->h_shard_mask = static_cast<uint8_t *>(q);
+            }
+        }
+    }
     A(&c->d_block_mask, B);
     A(&c->st, sizeof(SelState));
-    if (rc == SCAR_OK)
-        rc = plan_select(c);
-    const unsigned ng = c->sel_grid;
-    A(&c->ca.gt, ng * 4);
-    A(&c->ca.eq, ng * 4);
-    A(&c->ca.nf, ng * 4);
-    A(&c->ca.len_gt, ng * 8);
-    A(&c->ca.len_eq, ng * 8);
-    A(&c->rt_sum, nr * 8);
-    A(&c->rt_l1, nr * 8);
-    A(&c->rt_blocks, nr * 8);
-    A(&c->rt_elems, nr * 8);
+    if (rc == SCAR_OK) rc = plan_select(c);
+    // CTAs of the largest recovery / norm launch (segmented layouts reduce kReduceTile blocks per CTA: fewer)
+    const uint64_t max_ctas = recover_max_ctas(B, c->group_lanes);
+    c->norm_scratch_bytes = norm_scratch_words(max_ctas) * 8;
+    A(&c->norm_scratch, c->norm_scratch_bytes);
+    if (rc == SCAR_OK) c->rs = norm_scratch_at(c->norm_scratch, max_ctas);
     A(&c->cur.info, sizeof(SaveInfoDev));
     A(&c->d_norm, sizeof(NormInfoDev));
     if (rc == SCAR_OK && layout->block_offsets) A(&c->d_boff, (B + 1) * 8);
@@ -710,7 +827,7 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     // stream synchronisation at the end of init.
     std::vector<uint32_t> seg_block, wide;
     std::vector<uint64_t> seg_beg, seg_first;
-    if (rc == SCAR_OK && c->max_block_len > 2 * kSegElems) {
+    if (rc == SCAR_OK && long_blocks) {
         seg_first.resize(B + 1);
         for (uint64_t b = 0; b < B; ++b) {
             uint64_t beg, len;
@@ -738,7 +855,6 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
         A(&d_sbeg, ns * 8);
         A(&d_sfirst, (B + 1) * 8);
         A(&c->seg_part, ns * 8);
-        A(&c->selpos, B * 4);
         A(&c->wide_blocks, wide.size() * 4);
         c->n_wide_blocks = (unsigned)wide.size();
         if (rc == SCAR_OK && !wide.empty() &&
@@ -757,6 +873,7 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
         rc = SCAR_ERR_ALLOC;
     if (rc == SCAR_OK) {
         bool ok = cudaMemsetAsync(c->st, 0, sizeof(SelState), c->stream) == cudaSuccess &&
+                  cudaMemsetAsync(c->norm_scratch, 0xff, c->norm_scratch_bytes, c->stream) == cudaSuccess &&
                   cudaMemsetAsync(c->cur.info, 0, sizeof(SaveInfoDev), c->stream) == cudaSuccess &&
                   cudaMemsetAsync(c->d_norm, 0, sizeof(NormInfoDev), c->stream) == cudaSuccess &&
                   cudaMemsetAsync(c->score, 0, score_bytes ? score_bytes : 16, c->stream) == cudaSuccess &&
@@ -787,7 +904,7 @@ int scar_ckpt_block_scores(scar_ctx *c) {
     if (rc != SCAR_OK) return rc;
     c->last_call = 3;
     record(c, 0);
-    launch_scores(c);
+    launch_scores(c, nullptr);
     record(c, 1);
     CU_TRY(cudaGetLastError());
     return SCAR_OK;
@@ -916,13 +1033,8 @@ int scar_recover_partial_host(scar_ctx *c, void *h_x, const uint8_t *h_lost_shar
     std::vector<uint64_t> lo, hi;
     auto elem_of = [&](uint64_t b, uint64_t &e) -> int {
         if (b >= B) { e = c->g.n_elems; return SCAR_OK; }
-        if (c->g.boff) {
-            CU_TRY(cudaMemcpyAsync(&e, c->g.boff + b, 8, cudaMemcpyDeviceToHost, c->stream));
-            CU_TRY(cudaStreamSynchronize(c->stream));
-            return SCAR_OK;
-        }
-        uint64_t row = b / c->g.blocks_per_row, j = b % c->g.blocks_per_row;
-        e = row * c->g.row_len + j * c->g.block_elems;
+        uint64_t len;
+        host_range(c, b, e, len);
         return SCAR_OK;
     };
     for (uint64_t s = 0; s < S && B; ++s) {
@@ -973,10 +1085,9 @@ int scar_ckpt_selftest_arm_timeout(scar_ctx *c) {
     if (c->g.n_blocks == 0) return SCAR_ERR_STATE;
     int rc = check_device(c);
     if (rc != SCAR_OK) return rc;
-    // An arrival counter that starts just below zero wraps to a small number after the first arrivals and
-    // then never reaches the first barrier's target, so every CTA's wait runs out.
-    static const unsigned biased = 0u - 1u;
-    CU_TRY(cudaMemcpyAsync(&c->st->barrier, &biased, sizeof(unsigned), cudaMemcpyHostToDevice, c->stream));
+    // Host state only: the next selection is launched with waits that expect one arrival more than there are
+    // CTAs, so every one of them runs out.
+    c->arm_never = true;
     return SCAR_OK;
 }
 
@@ -1041,8 +1152,8 @@ int scar_ckpt_drain_enqueue(scar_ctx *c, uint64_t *ticket) {
     if (sl.state != 1) return SCAR_ERR_STATE;
     CU_TRY(cudaEventRecord(sl.saved, c->stream));
     CU_TRY(cudaStreamWaitEvent(c->drain_stream, sl.saved, 0));
-    // The payload length is only known on the device; k * (longest block) bounds it and is known here.
-    uint64_t elems = sl.k * c->max_block_len;
+    // The payload length is only known on the device; the k longest blocks bound it and are known here.
+    uint64_t elems = save_bound(c, sl.k);
     if (elems > c->drain_cap_elems) elems = c->drain_cap_elems;
     CU_TRY(cudaMemcpyAsync(sl.h_info, sl.dev.info, sizeof(SaveInfoDev), cudaMemcpyDeviceToHost, c->drain_stream));
     if (sl.k) CU_TRY(cudaMemcpyAsync(sl.h_sel, sl.dev.sel, sl.k * 4, cudaMemcpyDeviceToHost, c->drain_stream));
@@ -1106,17 +1217,6 @@ int scar_ckpt_drain_release(scar_ctx *c, uint64_t ticket) {
 namespace {
 
 constexpr size_t kIoStageBytes = 64u << 20;
-
-void host_range(const scar_ctx *c, uint64_t b, uint64_t &beg, uint64_t &len) {
-    if (!c->h_boff.empty()) {
-        beg = c->h_boff[b];
-        len = c->h_boff[b + 1] - beg;
-        return;
-    }
-    const uint64_t row = b / c->g.blocks_per_row, j = b % c->g.blocks_per_row, o = j * c->g.block_elems;
-    beg = row * c->g.row_len + o;
-    len = c->g.row_len - o < c->g.block_elems ? c->g.row_len - o : c->g.block_elems;
-}
 
 int write_all(int fd, const char *p, size_t n, uint64_t off) {
     while (n) {
@@ -1282,6 +1382,20 @@ int scar_ckpt_profile_read(scar_ctx *c, float ms[5]) {
         CU_TRY(cudaEventElapsedTime(&ms[4], c->ev[4], c->ev[5]));
     }
     return SCAR_OK;
+}
+
+int scar_ckpt_debug_select_stamps(scar_ctx *c, int64_t stamps[32]) {
+    if (!c || !stamps) return SCAR_ERR_INVALID_ARG;
+#ifdef SCAR_SELECT_STAMPS
+    static_assert(kSelStamps == 32, "size stated in scar.h");
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    CU_TRY(cudaStreamSynchronize(c->stream));
+    CU_TRY(cudaMemcpy(stamps, c->st->stamp, sizeof(long long) * kSelStamps, cudaMemcpyDeviceToHost));
+    return SCAR_OK;
+#else
+    return SCAR_ERR_STATE;
+#endif
 }
 
 int scar_ckpt_destroy(scar_ctx *c) {

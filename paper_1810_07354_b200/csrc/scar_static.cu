@@ -9,11 +9,11 @@
 // Such callers cannot create a scar_ctx, because scar_ckpt_init allocates the
 // checkpoint copy and its work arrays.
 //
-// The regular norm pass keeps one partial sum per block plus a few per-tile
-// sums and a ticket counter in memory that the context allocated.  Here that
-// scratch is a fixed array in the library's device image instead, so every GPU
-// that loads the library carries it (about 8 MiB) until the process exits, and
-// the block count is capped at SCAR_STATIC_MAX_BLOCKS.
+// The regular norm pass keeps one partial sum per CTA of its kernel, a few
+// per-tile sums and ticket counters in memory that the context allocated.  Here
+// that scratch is a fixed array in the library's device image instead, so every
+// GPU that loads the library carries it (about 0.4 MiB) until the process
+// exits, and the block count is capped at SCAR_STATIC_MAX_BLOCKS.
 #include <cstdint>
 #include <mutex>
 
@@ -26,11 +26,10 @@ using namespace scar;
 namespace {
 
 constexpr uint64_t kStaticMaxBlocks = SCAR_STATIC_MAX_BLOCKS;
-constexpr uint64_t kStaticMaxTiles = (kStaticMaxBlocks + kReduceTile - 1) / kReduceTile;
-// 8-byte words: one partial per block, four per-tile arrays, one word for the ticket.
-constexpr uint64_t kPartWords = kStaticMaxBlocks;
-constexpr uint64_t kTileWords = kStaticMaxTiles;
-constexpr uint64_t kScratchWords = kPartWords + 4 * kTileWords + 32;
+// The pass launches at most one CTA per kThreads / 4 blocks (the narrowest group has 4 lanes).
+constexpr uint64_t kStaticMaxCtas = kStaticMaxBlocks / (kThreads / 4) + 1;
+// 8-byte words: three slots per CTA, three per watcher.
+constexpr uint64_t kScratchWords = 3 * kStaticMaxCtas + 3 * kMaxWatchers;
 
 // In host code this name is only a handle for cudaGetSymbolAddress: it is not
 // a device address and must never be passed to a kernel as one.
@@ -64,27 +63,22 @@ static_assert(sizeof(NormInfoDev) == sizeof(scar_norm_info), "result layouts mus
 template <typename T>
 int run_static(const void *d_x, const void *d_z, const Geom &g, const LostSet &S, unsigned long long *scratch,
                scar_norm_info *d_out, cudaStream_t stream) {
-    using Sc = typename Elem<T>::score_t;
-    Sc *part = reinterpret_cast<Sc *>(scratch);
-    double *tile_sum = reinterpret_cast<double *>(scratch + kPartWords);
-    unsigned long long *tile_l1 = scratch + kPartWords + kTileWords;
-    unsigned long long *tile_blocks = scratch + kPartWords + 2 * kTileWords;
-    unsigned long long *tile_elems = scratch + kPartWords + 3 * kTileWords;
-    unsigned *ticket = reinterpret_cast<unsigned *>(scratch + kPartWords + 4 * kTileWords);
-    // The array keeps whatever the previous call left; only the ticket has to start at zero
-    // (every partial that is read is written first by this call).
-    if (cudaMemsetAsync(ticket, 0, sizeof(unsigned), stream) != cudaSuccess) return SCAR_ERR_CUDA;
-
     double units = (double)g.n_elems / (double)g.n_blocks;
     if (g.vec_ok) units /= 4.0;
     int G = 4;
     while (G < 32 && G * 4 < units) G <<= 1;
-    const unsigned grid = (G < 32 && S.mode == 2) ? (unsigned)((g.n_blocks + kThreads - 1) / kThreads)
-                                                  : (unsigned)((g.n_blocks + (kThreads / G) - 1) / (kThreads / G));
+    const RecoverShape sh = recover_shape(S.mode, S.n_work, G);
+    if (sh.grid > kStaticMaxCtas) return SCAR_ERR_CAPACITY;
+    const NormScratch rs = norm_scratch_at(scratch, sh.grid);
+    // Every call shares the array, and an earlier call may have laid it out for another grid size: the slots
+    // this call uses have to start out empty (all bits set).
+    if (cudaMemsetAsync(scratch, 0xff, norm_scratch_words(sh.grid) * 8, stream) != cudaSuccess) return SCAR_ERR_CUDA;
     T *x = static_cast<T *>(const_cast<void *>(d_x));  // the read-only instantiation never stores
     const T *z = static_cast<const T *>(d_z);
-#define SCAR_STATIC_LAUNCH(G_, VEC_) \
-    k_recover_blocks<T, kNormDefault, G_, VEC_, false><<<grid, kThreads, 0, stream>>>(x, z, g, S, nullptr, part)
+    NormInfoDev *out = reinterpret_cast<NormInfoDev *>(d_out);
+#define SCAR_STATIC_LAUNCH(G_, VEC_)                                                                            \
+    k_recover_blocks<T, kNormDefault, G_, VEC_, false><<<sh.grid, kThreads, 0, stream>>>(x, z, g, S, sh.chunk, \
+                                                                                       nullptr, rs, out)
     if (g.vec_ok) {
         if (G == 4) SCAR_STATIC_LAUNCH(4, true);
         else if (G == 8) SCAR_STATIC_LAUNCH(8, true);
@@ -97,9 +91,6 @@ int run_static(const void *d_x, const void *d_z, const Geom &g, const LostSet &S
         else SCAR_STATIC_LAUNCH(32, false);
     }
 #undef SCAR_STATIC_LAUNCH
-    const unsigned tiles = (unsigned)((g.n_blocks + kReduceTile - 1) / kReduceTile);
-    k_reduce_partials<T><<<tiles, kThreads, 0, stream>>>(part, g, S, tile_sum, tile_l1, tile_blocks, tile_elems, ticket,
-                                                        reinterpret_cast<NormInfoDev *>(d_out), true);
     return cudaGetLastError() == cudaSuccess ? SCAR_OK : SCAR_ERR_CUDA;
 }
 
@@ -112,6 +103,10 @@ extern "C" int scar_perturbation_norm_static(const void *d_x, const void *d_z, s
     if (layout->n_elems > 0 && (!d_x || !d_z)) return SCAR_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_z)) & 15) return SCAR_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // Looked up first, so that even a call on an empty layout is a complete warm-up of this device.
+    unsigned long long *scratch = nullptr;
+    int rc = scratch_on_current_device(&scratch);
+    if (rc != SCAR_OK) return rc;
     if (layout->n_elems == 0)
         return cudaMemsetAsync(d_out, 0, sizeof(scar_norm_info), stream) == cudaSuccess ? SCAR_OK : SCAR_ERR_CUDA;
     if (layout->block_elems == 0) return SCAR_ERR_LAYOUT;
@@ -136,9 +131,6 @@ extern "C" int scar_perturbation_norm_static(const void *d_x, const void *d_z, s
     S.mask = d_lost_blocks;
     S.n_work = g.n_blocks;
 
-    unsigned long long *scratch = nullptr;
-    int rc = scratch_on_current_device(&scratch);
-    if (rc != SCAR_OK) return rc;
     return dt == SCAR_F32 ? run_static<float>(d_x, d_z, g, S, scratch, d_out, stream)
                           : run_static<int>(d_x, d_z, g, S, scratch, d_out, stream);
 }

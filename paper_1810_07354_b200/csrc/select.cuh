@@ -9,62 +9,42 @@
 // such blocks rank first), or the uint64 l1 score itself.
 //
 // The whole selection is ONE kernel, launched cooperatively (every CTA is
-// resident), so its phases are separated by grid-wide barriers instead of
-// kernel boundaries: the score array is small (4-8 bytes per block), and five
-// to eight dependent launches cost more than the work itself.  Each CTA owns a
-// contiguous range of 2048-key tiles.
+// resident), because the score array is small (4-8 bytes per block) and a
+// chain of dependent launches costs more than the work itself.  Each CTA owns
+// a contiguous range of 4096-key tiles; when that range is a single tile (up
+// to about 600 000 blocks on a 148-SM device) its keys stay in registers from
+// the first load to the last store.  The CTAs meet at few points, and at each
+// of them a CTA pays for as few dependent trips to the L2 cache as possible:
 //
 //   digit passes   most-significant digit first: shared-memory histogram of
 //                  the keys that match the prefix so far, flushed with integer
-//                  atomics; barrier; every CTA resolves the digit from the
-//                  global histogram (the same small scan in every CTA).
-//                  Digits that are zero in every uint64 key are skipped.
-//   counts         with the threshold key tau and `need` (how many keys equal
-//                  to tau are taken): per-CTA counts and summed lengths of the
-//                  keys above / equal to tau; barrier; every CTA scans those
-//                  into its own output bases
-//   boundary       only when the tau-keys run out inside one CTA's range: that
-//                  CTA sums the lengths of the ones it takes; barrier
+//                  atomics; one arrival counter per pass (fire-and-forget
+//                  increment, then an acquiring poll); every CTA resolves the
+//                  digit from the global histogram (the same small scan in
+//                  every CTA).  Digits that are zero in every uint64 key are
+//                  skipped.
+//   exchange       with the threshold key tau and `need` (how many keys equal
+//                  to tau are taken) every CTA publishes one record: how many
+//                  of its keys lie above / at tau and their summed lengths.
+//                  Thread c of every CTA waits for the record of CTA c, and a
+//                  CTA-wide scan of the records gives the CTA its output bases
+//                  and the totals.  This one step stands for a barrier, the
+//                  per-CTA counts and their prefix sums.
+//   boundary       only when the tau-keys run out inside one CTA's range and
+//                  block lengths differ: the CTAs after it recompute, from that
+//                  CTA's keys, the summed length of the tau-blocks it takes
 //   emit           ordered compaction into sel[] / poff[]
 //
-// The barrier is a counter in global memory with a bounded spin: a CTA that
-// gives up records an error and leaves, and the host reports SCAR_ERR_TIMEOUT.
+// Every wait is bounded: a CTA that gives up records an error and leaves, the
+// others see it and leave too, and the host reports SCAR_ERR_TIMEOUT.  The
+// counters, histograms and records must be zero when the kernel starts
+// (sel_state_clear, run by the kernel that precedes it on the stream, or a
+// memset); the kernel never has to put them back.
 #pragma once
 #include "block_pass.cuh"
+#include "sel_state.cuh"
 
 namespace scar {
-
-constexpr int kMaxPasses = 6;
-constexpr int kHistBins = 2048;
-constexpr int kSelTile = 2048;  // keys per tile
-constexpr int kPerThread = kSelTile / kThreads;
-constexpr unsigned kBarrierSpinLimit = 1u << 21;  // each try is a global load and a short sleep: gives up after >= 0.1 s
-
-struct SelState {
-    unsigned long long key_or;  // OR of all uint64 keys seen since the last selection
-    unsigned long long partial_len;  // summed length of the tau-blocks taken in the boundary CTA
-    unsigned barrier;           // arrivals at the grid barrier during the running selection
-    unsigned departed;          // CTAs that have passed their last barrier
-    unsigned error;             // non-zero once a barrier wait gave up
-    unsigned ticket_reduce;     // ticket of the perturbation-norm reduction (block_pass.cuh)
-    unsigned hist[kMaxPasses][kHistBins];
-};
-
-struct SaveInfoDev {
-    unsigned long long k;
-    unsigned long long payload_elems;
-    unsigned long long nonfinite_blocks;
-    unsigned long long error;  // copy of SelState::error at the end of the selection
-};
-
-// One entry per CTA of the selection kernel.
-struct CtaArrays {
-    unsigned *gt;               // keys > tau
-    unsigned *eq;               // keys == tau
-    unsigned *nf;               // non-finite scores
-    unsigned long long *len_gt; // summed block lengths of the above
-    unsigned long long *len_eq;
-};
 
 // Digit plan per key width: 11/11/10 bits for 32-bit keys, 11/11/11/11/10/10 for 64-bit keys.
 template <typename K> struct KeyTraits;
@@ -104,32 +84,8 @@ template <> struct ScoreKey<unsigned> {  // caller-supplied 32-bit priorities (r
     static __device__ __forceinline__ bool nonfinite(K) { return false; }
 };
 
-// Exclusive prefix sum of one value per thread over the CTA; *total gets the sum.
-template <typename W> __device__ __forceinline__ W cta_excl_scan(W v, W *sh /*kThreads/32 + 1*/, W *total) {
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    W inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        W n = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += n;
-    }
-    __syncthreads();
-    if (lane == 31) sh[w] = inc;
-    __syncthreads();
-    W before = 0, all = 0;
-#pragma unroll
-    for (int i = 0; i < kThreads / 32; ++i) {
-        W t = sh[i];
-        if (i < w) before += t;
-        all += t;
-    }
-    if (total) *total = all;
-    return before + inc - v;
-}
-
-// Sums N values per thread over the CTA with one pair of barriers (the selection kernel is a chain of
-// short dependent phases, so barriers are what it pays for).  sh holds N * kThreads / 32 words.
-template <int N>
+// Sums N values per thread over the CTA with one pair of barriers.  sh holds N * NT / 32 words.
+template <int N, int NT = kThreads>
 __device__ __forceinline__ void cta_sum_n(unsigned long long (&v)[N], unsigned long long *sh) {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
 #pragma unroll
@@ -144,40 +100,54 @@ __device__ __forceinline__ void cta_sum_n(unsigned long long (&v)[N], unsigned l
     for (int i = 0; i < N; ++i) {
         unsigned long long t = 0;
 #pragma unroll
-        for (int j = 0; j < kThreads / 32; ++j) t += sh[j * N + i];
+        for (int j = 0; j < NT / 32; ++j) t += sh[j * N + i];
         v[i] = t;
     }
 }
 
-// Grid-wide barrier number `phase` (1, 2, ...) of a cooperative launch: every
-// CTA of the grid must call it the same number of times.  Returns false when
-// the wait was abandoned (it cannot happen while all CTAs are resident, which a
+__device__ __forceinline__ unsigned ld_acquire(const unsigned *p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(__cvta_generic_to_global(p)) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(unsigned *p, unsigned v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(__cvta_generic_to_global(p)), "r"(v) : "memory");
+}
+
+// Polls *word until it reaches target.  False when the wait was abandoned: after kSpinLimit polls, or as soon
+// as another CTA has recorded an error.
+__device__ __forceinline__ bool spin_until_at_least(const unsigned *word, unsigned target, const SelState *st) {
+    unsigned tries = 0;
+    while (ld_acquire(word) < target) {
+        ++tries;
+        if (tries > kSpinLimit || ((tries & 255u) == 0 && ld_acquire(&st->error) != 0)) return false;
+        if (tries > 16) __nanosleep(tries > 4096 ? 256 : 32);
+    }
+    return true;
+}
+
+__device__ __forceinline__ void sel_fail(SelState *st, SaveInfoDev *info) {
+    atomicExch(&st->error, 1u);
+    *reinterpret_cast<volatile unsigned long long *>(&info->error) = 1ull;
+    __threadfence();
+}
+
+// Arrival at the meeting point after a digit pass: every CTA adds one to *ctr and waits until `target` CTAs
+// have.  What the CTA's threads wrote before (their histogram updates) is visible to every CTA that gets past
+// the wait.  Returns false when the wait was abandoned (it cannot happen while all CTAs are resident, which a
 // cooperative launch guarantees; the bound is there so that nothing can hang).
-__device__ __forceinline__ bool grid_barrier(SelState *st, unsigned phase) {
-    __shared__ bool ok;
+__device__ __forceinline__ bool sel_arrive_wait(unsigned *ctr, unsigned target, SelState *st, SaveInfoDev *info,
+                                                int *sh_ok) {
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
-        const unsigned target = phase * gridDim.x;
-        bool good = true;
-        if (atomicAdd(&st->barrier, 1u) + 1 < target) {  // the last CTA to arrive does not wait
-            volatile unsigned *ctr = &st->barrier;
-            volatile unsigned *err = &st->error;
-            unsigned tries = 0;
-            while (*ctr < target) {
-                if (++tries > kBarrierSpinLimit || ((tries & 1023u) == 0 && *err != 0)) {
-                    atomicExch(&st->error, 1u);
-                    good = false;
-                    break;
-                }
-                __nanosleep(32);
-            }
-        }
-        __threadfence();
-        ok = good;
+        atomicAdd(ctr, 1u);  // result unused: a reduction, nothing to wait for
+        const bool good = spin_until_at_least(ctr, target, st);
+        if (!good) sel_fail(st, info);
+        *sh_ok = good;
     }
     __syncthreads();
-    return ok;
+    return *sh_ok != 0;
 }
 
 // Resolves one digit: scanning bins from the highest down, finds the bin d with
@@ -187,19 +157,26 @@ template <int WIDTH>
 __device__ __forceinline__ unsigned resolve_digit_w(const unsigned *hist, unsigned long long &remaining,
                                                     unsigned long long *sh_scan, unsigned long long *sh_out) {
     constexpr int nb = 1 << WIDTH;
-    constexpr int per = nb / kThreads;  // 8 or 4: a compile-time count, so all loads are in flight together
+    constexpr int per = nb / kSelThreads;  // 4 or 2 consecutive bins per thread, highest bins in thread 0
+    static_assert(per == 4 || per == 2, "one vector load per thread");
     unsigned local[per];
+    const unsigned *src = hist + (nb - (int)(threadIdx.x + 1) * per);
+    if (per == 4) {
+        const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(src));
+        local[0] = v.w; local[1] = v.z; local[per - 2] = v.y; local[per - 1] = v.x;
+    } else {
+        const uint2 v = __ldcg(reinterpret_cast<const uint2 *>(src));
+        local[0] = v.y; local[1] = v.x;
+    }
     unsigned long long sum = 0;
 #pragma unroll
-    for (int i = 0; i < per; ++i) local[i] = __ldcg(hist + (nb - 1 - (threadIdx.x * per + i)));
-#pragma unroll
     for (int i = 0; i < per; ++i) sum += local[i];
-    unsigned long long cum = cta_excl_scan<unsigned long long>(sum, sh_scan, nullptr);
+    unsigned long long cum = cta_excl_scan<unsigned long long, kSelThreads>(sum, sh_scan, nullptr);
 #pragma unroll
     for (int i = 0; i < per; ++i) {
         unsigned long long h = local[i];
         if (cum < remaining && remaining <= cum + h) {
-            sh_out[0] = (unsigned long long)(nb - 1 - (threadIdx.x * per + i));
+            sh_out[0] = (unsigned long long)(nb - 1 - ((int)threadIdx.x * per + i));
             sh_out[1] = remaining - cum;
         }
         cum += h;
@@ -217,52 +194,119 @@ __device__ __forceinline__ unsigned resolve_digit(const unsigned *hist, int widt
                        : resolve_digit_w<10>(hist, remaining, sh_scan, sh_out);
 }
 
-// Flags of the kPerThread consecutive blocks a thread owns in tile t.
+// Keys of the kSelPerThread consecutive blocks a thread owns in a tile (first = index of the first of them);
+// bit j of valid says block first + j exists.
 template <typename S>
-__device__ __forceinline__ void tile_flags(const S *__restrict__ score, unsigned long long n_blocks, unsigned t, bool none,
-                                           typename ScoreKey<S>::K tau, unsigned &gt_bits, unsigned &eq_bits,
-                                           unsigned &nf_bits) {
+__device__ __forceinline__ void load_keys(const S *__restrict__ score, unsigned long long n_blocks,
+                                          unsigned long long first, typename ScoreKey<S>::K (&key)[kSelPerThread],
+                                          unsigned &valid) {
     using SK = ScoreKey<S>;
-    using K = typename SK::K;
-    gt_bits = eq_bits = nf_bits = 0;
-    const unsigned long long first = (unsigned long long)t * kSelTile + (unsigned long long)threadIdx.x * kPerThread;
+    static_assert(kSelPerThread == 8 && (sizeof(S) == 4 || sizeof(S) == 8), "vector loads below");
+    if (first + kSelPerThread <= n_blocks && (reinterpret_cast<uintptr_t>(score) & 15) == 0) {
+        S raw[kSelPerThread];
+        uint4 *dst = reinterpret_cast<uint4 *>(raw);
+        const uint4 *src = reinterpret_cast<const uint4 *>(score + first);
 #pragma unroll
-    for (int j = 0; j < kPerThread; ++j) {
-        unsigned long long b = first + j;
-        if (b < n_blocks) {
-            K key = SK::key(score[b]);
-            if (SK::nonfinite(key)) nf_bits |= 1u << j;
-            if (!none) {
-                if (key > tau) gt_bits |= 1u << j;
-                else if (key == tau) eq_bits |= 1u << j;
-            }
+        for (int i = 0; i < (int)(sizeof(S) * kSelPerThread / 16); ++i) dst[i] = src[i];
+#pragma unroll
+        for (int j = 0; j < kSelPerThread; ++j) key[j] = SK::key(raw[j]);
+        valid = 0xffu;
+        return;
+    }
+    valid = 0;
+#pragma unroll
+    for (int j = 0; j < kSelPerThread; ++j) {
+        key[j] = 0;
+        if (first + j < n_blocks) {
+            key[j] = SK::key(score[first + j]);
+            valid |= 1u << j;
         }
     }
 }
 
+// Length of every block of an implicit layout when they are all the same, else 0.
+__device__ __forceinline__ unsigned long long uniform_block_len(const Geom &g) {
+    if (g.boff) return 0;
+    if (g.blocks_per_row == 1) return g.row_len;
+    return g.row_len % g.block_elems == 0 ? (unsigned long long)g.block_elems : 0ull;
+}
+
+// Summed length of the first `take` blocks (in id order) of CTA cb's tile range whose key equals tau.
 template <typename S>
-__global__ void __launch_bounds__(kThreads)
-k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st, CtaArrays ca, SaveInfoDev *info,
-         uint32_t *__restrict__ sel, unsigned long long *__restrict__ poff, unsigned n_tiles, unsigned tiles_per_cta) {
+__device__ __forceinline__ unsigned long long boundary_len(const S *__restrict__ score, const Geom &g, unsigned cb,
+                                                           unsigned tiles_per_cta, unsigned n_tiles,
+                                                           typename ScoreKey<S>::K tau, unsigned long long take,
+                                                           unsigned long long *sh_scan, unsigned long long *sh_red) {
+    typedef unsigned long long u64;
+    using K = typename ScoreKey<S>::K;
+    const u64 ulen = uniform_block_len(g);
+    if (ulen) return take * ulen;
+    const unsigned t_lo = cb * tiles_per_cta;
+    const unsigned t_hi = t_lo + tiles_per_cta < n_tiles ? t_lo + tiles_per_cta : n_tiles;
+    u64 run = 0;
+    u64 pl[1] = {0};
+    for (unsigned t = t_lo; t < t_hi; ++t) {
+        K key[kSelPerThread];
+        unsigned valid;
+        const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kSelPerThread;
+        load_keys<S>(score, g.n_blocks, first, key, valid);
+        unsigned eq_bits = 0;
+#pragma unroll
+        for (int j = 0; j < kSelPerThread; ++j)
+            if ((valid >> j & 1u) && key[j] == tau) eq_bits |= 1u << j;
+        u64 tot;
+        u64 rank = run + cta_excl_scan<u64, kSelThreads>(__popc(eq_bits), sh_scan, &tot);
+        run += tot;
+        for (int j = 0; j < kSelPerThread; ++j)
+            if (eq_bits >> j & 1u) {
+                if (rank < take) {
+                    uint64_t beg, len;
+                    g.range((uint32_t)(first + j), beg, len);
+                    pl[0] += len;
+                }
+                ++rank;
+            }
+    }
+    cta_sum_n<1, kSelThreads>(pl, sh_red);
+    return pl[0];
+}
+
+// REG: every CTA owns exactly one tile and keeps its keys in registers.  never != 0 (self-test only) makes every
+// wait expect one arrival more than there are CTAs, so that it runs out.
+template <typename S, bool REG>
+__global__ void __launch_bounds__(kSelThreads, 1)
+k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st, SaveInfoDev *info,
+         uint32_t *__restrict__ sel, unsigned long long *__restrict__ poff, unsigned n_tiles, unsigned tiles_per_cta,
+         unsigned never) {
     using SK = ScoreKey<S>;
     using K = typename SK::K;
     using KT = KeyTraits<K>;
     typedef unsigned long long u64;
     __shared__ unsigned sh_hist[kHistBins];
-    __shared__ u64 sh_scan[kThreads / 32 + 1];
+    __shared__ u64 sh_scan[kSelThreads / 32];
     __shared__ u64 sh_out[2];
-    __shared__ u64 sh_red[6 * kThreads / 32];
-    __shared__ long long sh_boundary;
+    __shared__ u64 sh_red[6 * kSelThreads / 32];
+    __shared__ int sh_boundary;
     __shared__ u64 sh_boundary_take;
-    __shared__ bool sh_last;
+    __shared__ int sh_ok;
 
     griddep_launch();  // the pack kernel may be scheduled while this one runs; it waits before reading sel / poff
+    SEL_STAMP(st, 0);
     const u64 B = g.n_blocks;
     const unsigned t_lo = blockIdx.x * tiles_per_cta;
     const unsigned t_hi = t_lo + tiles_per_cta < n_tiles ? t_lo + tiles_per_cta : n_tiles;
     const bool none = k == 0;
-    const u64 key_or = KT::kSkippable ? st->key_or : ~0ull;  // reset only after the last barrier
-    unsigned phase = 0;
+    const u64 key_or = KT::kSkippable ? st->key_or : ~0ull;  // put back to 0 after the exchange
+    K key[kSelPerThread];
+    unsigned valid = 0;
+    if (REG) load_keys<S>(score, B, (u64)t_lo * kSelTile + (u64)threadIdx.x * kSelPerThread, key, valid);
+    for (int i = threadIdx.x; i < kHistBins; i += kSelThreads) sh_hist[i] = 0;
+    if (threadIdx.x == 0) {
+        sh_boundary = -1;
+        sh_boundary_take = 0;
+    }
+    __syncthreads();
+    SEL_STAMP(st, 1);  // keys loaded
     bool alive = true;
 
     // ---- digit passes: tau = the k-th largest key, need = how many keys equal to tau are taken
@@ -275,154 +319,143 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
                 prefix <<= width;
                 continue;
             }
-            for (int i = threadIdx.x; i < kHistBins; i += kThreads) sh_hist[i] = 0;
-            __syncthreads();
             for (unsigned t = t_lo; t < t_hi; ++t) {
-                const u64 base = (u64)t * kSelTile;
+                if (!REG) load_keys<S>(score, B, (u64)t * kSelTile + (u64)threadIdx.x * kSelPerThread, key, valid);
 #pragma unroll
-                for (int j = 0; j < kPerThread; ++j) {
-                    const u64 i = base + threadIdx.x + (u64)j * kThreads;
-                    if (i < B) {
-                        const K key = SK::key(score[i]);
-                        const bool match = p == 0 || ((u64)key >> (shift + width)) == prefix;
-                        if (match) atomicAdd(&sh_hist[(unsigned)(((u64)key >> shift) & mask)], 1u);
-                    }
+                for (int j = 0; j < kSelPerThread; ++j) {
+                    const bool match = p == 0 || ((u64)key[j] >> (shift + width)) == prefix;
+                    if ((valid >> j & 1u) && match) atomicAdd(&sh_hist[(unsigned)(((u64)key[j] >> shift) & mask)], 1u);
                 }
             }
             __syncthreads();
-            for (int i = threadIdx.x; i < (1 << width); i += kThreads) {
+            SEL_STAMP(st, 2 + 4 * p);  // pass p: shared histogram built
+            for (int i = threadIdx.x; i < (1 << width); i += kSelThreads) {
                 const unsigned c = sh_hist[i];
-                if (c) atomicAdd(&st->hist[p][i], c);
+                if (c) {
+                    atomicAdd(&st->hist[p][i], c);
+                    sh_hist[i] = 0;  // ready for the next pass
+                }
             }
-            alive = grid_barrier(st, ++phase);
+            SEL_STAMP(st, 3 + 4 * p);  // flushed
+            alive = sel_arrive_wait(&st->arrive[p], gridDim.x + never, st, info, &sh_ok);
+            SEL_STAMP(st, 4 + 4 * p);  // every CTA has arrived
             if (alive) prefix = (prefix << width) | resolve_digit(st->hist[p], width, need, sh_scan, sh_out);
+            SEL_STAMP(st, 5 + 4 * p);  // digit resolved
         }
     }
     const K tau = (K)prefix;
 
-    // ---- counts over this CTA's tiles
-    u64 c_gt = 0, c_eq = 0, c_nf = 0, lgt = 0, leq = 0;
+    // ---- this CTA's record: counts and summed lengths of its keys above / at tau
     if (alive) {
+        u64 five[5] = {0, 0, 0, 0, 0};  // c_gt, c_eq, c_nf, len_gt, len_eq
         for (unsigned t = t_lo; t < t_hi; ++t) {
-            unsigned gt_bits, eq_bits, nf_bits;
-            tile_flags<S>(score, B, t, none, tau, gt_bits, eq_bits, nf_bits);
-            const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kPerThread;
-            for (int j = 0; j < kPerThread; ++j)
-                if ((gt_bits | eq_bits) >> j & 1u) {
-                    uint64_t beg, len;
-                    g.range((uint32_t)(first + j), beg, len);
-                    if (gt_bits >> j & 1u) lgt += len;
-                    else leq += len;
+            const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kSelPerThread;
+            if (!REG) load_keys<S>(score, B, first, key, valid);
+#pragma unroll
+            for (int j = 0; j < kSelPerThread; ++j) {
+                if (!(valid >> j & 1u)) continue;
+                if (SK::nonfinite(key[j])) ++five[2];
+                if (none || key[j] < tau) continue;
+                uint64_t beg, len;
+                g.range((uint32_t)(first + j), beg, len);
+                if (key[j] > tau) {
+                    ++five[0];
+                    five[3] += len;
+                } else {
+                    ++five[1];
+                    five[4] += len;
                 }
-            c_gt += __popc(gt_bits);
-            c_eq += __popc(eq_bits);
-            c_nf += __popc(nf_bits);
+            }
         }
-        u64 five[5] = {c_gt, c_eq, c_nf, lgt, leq};
-        cta_sum_n<5>(five, sh_red);
-        c_gt = five[0], c_eq = five[1], c_nf = five[2], lgt = five[3], leq = five[4];
+        cta_sum_n<5, kSelThreads>(five, sh_red);
+        SEL_STAMP(st, 26);  // own counts known
         if (threadIdx.x == 0) {
-            ca.gt[blockIdx.x] = (unsigned)c_gt;
-            ca.eq[blockIdx.x] = (unsigned)c_eq;
-            ca.nf[blockIdx.x] = (unsigned)c_nf;
-            ca.len_gt[blockIdx.x] = lgt;
-            ca.len_eq[blockIdx.x] = leq;
-            sh_boundary = -1;
-            sh_boundary_take = 0;
+            SelRecord *r = &st->rec[blockIdx.x];
+            r->c_gt = (unsigned)five[0];
+            r->c_eq = (unsigned)five[1];
+            r->c_nf = (unsigned)five[2];
+            r->len_gt = five[3];
+            r->len_eq = five[4];
+            __threadfence();
+            st_release(&r->ready, 1u);
         }
-        alive = grid_barrier(st, ++phase);
     }
 
-    // ---- every CTA scans the per-CTA counts into its own bases (the same scan in every CTA)
+    // ---- exchange: thread c takes the record of CTA c; one scan gives this CTA its bases and the totals
     u64 my_eq_before = 0, my_sel_base = 0, my_len_base = 0, total_n = 0, total_l = 0, total_nf = 0;
-    long long cb = -1;
+    int cb = -1;
     if (alive) {
-        u64 carry = 0, a_eq = 0, a_n = 0, a_l = 0, t_n = 0, t_l = 0, t_nf = 0;
-        for (unsigned c0 = 0; c0 < gridDim.x; c0 += kThreads) {
-            const unsigned c = c0 + threadIdx.x;
-            const bool in = c < gridDim.x;
-            const u64 e = in ? __ldcg(ca.eq + c) : 0;
-            u64 tot;
-            const u64 ex = carry + cta_excl_scan<u64>(e, sh_scan, &tot);
-            carry += tot;
-            if (in) {
-                u64 take = need > ex ? need - ex : 0;
-                if (take > e) take = e;
-                if (take != 0 && take != e) {  // the tau-keys run out inside this CTA's range
-                    sh_boundary = c;
-                    sh_boundary_take = take;
-                }
-                const u64 n = __ldcg(ca.gt + c) + take;
-                const u64 l = __ldcg(ca.len_gt + c) + (take == e ? __ldcg(ca.len_eq + c) : 0);
-                t_n += n;
-                t_l += l;
-                t_nf += __ldcg(ca.nf + c);
-                if (c < blockIdx.x) {
-                    a_eq += e;
-                    a_n += n;
-                    a_l += l;
-                }
+        const unsigned c = threadIdx.x;
+        u64 e = 0, gt = 0, nf = 0, lg = 0, le = 0;
+        bool ok = true;
+        if (c < gridDim.x + never) {
+            const SelRecord *r = &st->rec[c];
+            ok = spin_until_at_least(&r->ready, 1u, st);
+            if (!ok) {
+                sel_fail(st, info);
+            } else if (c < gridDim.x) {
+                e = __ldcg(&r->c_eq);
+                gt = __ldcg(&r->c_gt);
+                nf = __ldcg(&r->c_nf);
+                lg = __ldcg(&r->len_gt);
+                le = __ldcg(&r->len_eq);
             }
         }
-        u64 six[6] = {a_eq, a_n, a_l, t_n, t_l, t_nf};
-        cta_sum_n<6>(six, sh_red);
-        my_eq_before = six[0], my_sel_base = six[1], my_len_base = six[2];
-        total_n = six[3], total_l = six[4], total_nf = six[5];
-        cb = sh_boundary;  // written before the barriers inside cta_sum_n
-    }
-
-    // ---- boundary CTA: summed length of the tau-blocks it takes (lowest ids first)
-    if (alive && cb >= 0) {  // the same decision in every CTA
-        if ((long long)blockIdx.x == cb) {
-            const u64 take = sh_boundary_take;
-            u64 run = 0, pl = 0;
-            for (unsigned t = t_lo; t < t_hi; ++t) {
-                unsigned gt_bits, eq_bits, nf_bits;
-                tile_flags<S>(score, B, t, false, tau, gt_bits, eq_bits, nf_bits);
-                u64 tot;
-                u64 rank = run + cta_excl_scan<u64>(__popc(eq_bits), sh_scan, &tot);
-                run += tot;
-                const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kPerThread;
-                for (int j = 0; j < kPerThread; ++j)
-                    if (eq_bits >> j & 1u) {
-                        if (rank < take) {
-                            uint64_t beg, len;
-                            g.range((uint32_t)(first + j), beg, len);
-                            pl += len;
-                        }
-                        ++rank;
-                    }
-            }
-            pl = cta_sum<u64>(pl, sh_red);
-            if (threadIdx.x == 0) st->partial_len = pl;
-        }
-        alive = grid_barrier(st, ++phase);
+        alive = __syncthreads_and(ok) != 0;
+        SEL_STAMP(st, 27);  // every CTA's record read
         if (alive) {
-            const u64 pl = __ldcg(&st->partial_len);
-            total_l += pl;
-            if ((long long)blockIdx.x > cb) my_len_base += pl;
+            const u64 ex = cta_excl_scan<u64, kSelThreads>(e, sh_scan, nullptr);
+            u64 take = need > ex ? need - ex : 0;
+            if (take > e) take = e;
+            if (take != 0 && take != e) {  // the tau-keys run out inside CTA c's range
+                sh_boundary = (int)c;
+                sh_boundary_take = take;
+            }
+            const u64 n = gt + take;
+            const u64 l = lg + (take == e ? le : 0);
+            const bool mine = c < blockIdx.x;
+            u64 six[6] = {mine ? e : 0, mine ? n : 0, mine ? l : 0, n, l, nf};
+            cta_sum_n<6, kSelThreads>(six, sh_red);
+            my_eq_before = six[0], my_sel_base = six[1], my_len_base = six[2];
+            total_n = six[3], total_l = six[4], total_nf = six[5];
+            cb = sh_boundary;  // written before the barriers inside cta_sum_n
         }
     }
 
+    // ---- boundary: the CTAs behind the one where the tau-keys run out need the length of what it takes
+    if (alive && cb >= 0 && (int)blockIdx.x >= cb) {
+        const u64 pl = boundary_len<S>(score, g, (unsigned)cb, tiles_per_cta, n_tiles, tau, sh_boundary_take, sh_scan,
+                                       sh_red);
+        total_l += pl;
+        if ((int)blockIdx.x > cb) my_len_base += pl;
+    }
+
+    SEL_STAMP(st, 28);  // bases known
     // ---- emit: ordered compaction of this CTA's tiles
     if (alive && !none) {
         u64 run_eq = my_eq_before, pos_base = my_sel_base, off_base = my_len_base;
         for (unsigned t = t_lo; t < t_hi; ++t) {
-            unsigned gt_bits, eq_bits, nf_bits;
-            tile_flags<S>(score, B, t, false, tau, gt_bits, eq_bits, nf_bits);
-            u64 tot_eq, tot_n, tot_l;
-            u64 rank = run_eq + cta_excl_scan<u64>(__popc(eq_bits), sh_scan, &tot_eq);
+            const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kSelPerThread;
+            if (!REG) load_keys<S>(score, B, first, key, valid);
+            unsigned gt_bits = 0, eq_bits = 0;
+#pragma unroll
+            for (int j = 0; j < kSelPerThread; ++j)
+                if (valid >> j & 1u) {
+                    if (key[j] > tau) gt_bits |= 1u << j;
+                    else if (key[j] == tau) eq_bits |= 1u << j;
+                }
+            u64 tot_eq;
+            u64 rank = run_eq + cta_excl_scan<u64, kSelThreads>(__popc(eq_bits), sh_scan, &tot_eq);
             unsigned take_bits = gt_bits;
-            for (int j = 0; j < kPerThread; ++j)
+            for (int j = 0; j < kSelPerThread; ++j)
                 if (eq_bits >> j & 1u) {
                     if (rank < need) take_bits |= 1u << j;
                     ++rank;
                 }
-            const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kPerThread;
-            u64 lens[kPerThread];
+            u64 lens[kSelPerThread];
             u64 lsum = 0;
 #pragma unroll
-            for (int j = 0; j < kPerThread; ++j) {
+            for (int j = 0; j < kSelPerThread; ++j) {
                 lens[j] = 0;
                 if (take_bits >> j & 1u) {
                     uint64_t beg, len;
@@ -431,16 +464,15 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
                     lsum += len;
                 }
             }
-            // one scan for both outputs: block counts in the top 16 bits (at most 2048 per tile), summed
+            // one scan for both outputs: block counts in the top 16 bits (at most 4096 per tile), summed
             // lengths below (a buffer has fewer than 2^48 elements: init rejects more)
             u64 tot_both;
-            const u64 both = cta_excl_scan<u64>(((u64)__popc(take_bits) << 48) | lsum, sh_scan, &tot_both);
+            const u64 both =
+                cta_excl_scan<u64, kSelThreads>(((u64)__popc(take_bits) << 48) | lsum, sh_scan, &tot_both);
             u64 pos = pos_base + (both >> 48);
             u64 off = off_base + (both & ((1ull << 48) - 1));
-            tot_n = tot_both >> 48;
-            tot_l = tot_both & ((1ull << 48) - 1);
 #pragma unroll
-            for (int j = 0; j < kPerThread; ++j)
+            for (int j = 0; j < kSelPerThread; ++j)
                 if (take_bits >> j & 1u) {
                     sel[pos] = (uint32_t)(first + j);
                     poff[pos] = off;
@@ -448,39 +480,328 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
                     off += lens[j];
                 }
             run_eq += tot_eq;
-            pos_base += tot_n;
-            off_base += tot_l;
+            pos_base += tot_both >> 48;
+            off_base += tot_both & ((1ull << 48) - 1);
         }
     }
-    if (alive && blockIdx.x == 0 && threadIdx.x == 0) {
+    SEL_STAMP(st, 29);  // emitted
+    // The last CTA lies behind every boundary, so its totals are complete.  By now every CTA has read key_or.
+    if (alive && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {
         info->k = total_n;
         info->payload_elems = total_l;
         info->nonfinite_blocks = total_nf;
         poff[total_n] = total_l;
+        if (KT::kSkippable) st->key_or = 0;  // forget which uint64 key bits were seen
+    }
+}
+
+// ---- the same selection when every CTA owns exactly one tile -----------------------
+//
+// This is the form that runs for up to kSelTile * (number of SMs) blocks.  The kernel is a chain of short
+// phases that each run once, so its time is latency: trips to L2, CTA barriers, and fetching code that has not
+// run yet.  Hence: a thread's keys sit in (padded, conflict-free) shared memory and the loops over them are not
+// unrolled, which keeps the code short; counts travel as 32-bit words and are added with the warp-reduce
+// instruction; one packed scan over the CTAs' records gives all prefix sums; and layouts whose blocks all have
+// one length skip every sum of lengths.
+template <int WIDTH>
+__device__ __forceinline__ unsigned resolve_digit32_w(const unsigned *hist, unsigned &remaining, unsigned *sh_scan,
+                                                      unsigned *sh_out) {
+    constexpr int nb = 1 << WIDTH;
+    constexpr int per = nb / kSelThreads;  // 4 or 2 consecutive bins per thread, highest bins in thread 0
+    unsigned local[4] = {0, 0, 0, 0};
+    const unsigned *src = hist + (nb - (int)(threadIdx.x + 1) * per);
+    if (per == 4) {
+        const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(src));
+        local[0] = v.w, local[1] = v.z, local[2] = v.y, local[3] = v.x;
+    } else {
+        const uint2 v = __ldcg(reinterpret_cast<const uint2 *>(src));
+        local[0] = v.y, local[1] = v.x;
+    }
+    const unsigned sum = (local[0] + local[1]) + (local[2] + local[3]);
+    unsigned cum = cta_excl_scan<unsigned, kSelThreads>(sum, sh_scan, nullptr);
+#pragma unroll
+    for (int i = 0; i < per; ++i) {
+        const unsigned h = local[i];
+        if (cum < remaining && remaining <= cum + h) {
+            sh_out[0] = (unsigned)(nb - 1 - ((int)threadIdx.x * per + i));
+            sh_out[1] = remaining - cum;
+        }
+        cum += h;
+    }
+    __syncthreads();
+    remaining = sh_out[1];
+    return sh_out[0];  // the next write to sh_out comes after further barriers
+}
+
+template <typename S>
+__global__ void __launch_bounds__(kSelThreads, 1)
+k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, SaveInfoDev *info,
+              uint32_t *__restrict__ sel, unsigned long long *__restrict__ poff, unsigned never) {
+    using SK = ScoreKey<S>;
+    using K = typename SK::K;
+    using KT = KeyTraits<K>;
+    typedef unsigned long long u64;
+    constexpr int P = kSelPerThread, kPad = P + 1;  // odd stride: the threads of a warp hit 32 different banks
+    constexpr int kWarps = kSelThreads / 32;
+    __shared__ K sh_key[kSelThreads * kPad];
+    __shared__ unsigned sh_hist[kHistBins];
+    __shared__ unsigned sh_scan[kWarps];
+    __shared__ u64 sh_scan64[kWarps];
+    __shared__ unsigned sh_out[2];
+    __shared__ unsigned sh_w[kWarps];
+    __shared__ u64 sh_wl[2 * kWarps];
+    __shared__ u64 sh_mine[3];
+    __shared__ int sh_boundary;
+    __shared__ unsigned sh_boundary_take;
+    __shared__ int sh_ok;
+
+    griddep_launch();  // the pack kernel may be scheduled while this one runs; it waits before reading sel / poff
+    SEL_STAMP(st, 0);
+    const unsigned B = (unsigned)g.n_blocks;  // fewer than 2^32 blocks: init rejects more
+    const unsigned first = blockIdx.x * kSelTile + threadIdx.x * P;
+    const bool none = k == 0;
+    const u64 key_or = KT::kSkippable ? st->key_or : ~0ull;  // put back to 0 after the exchange
+    const u64 ulen = uniform_block_len(g);
+    K *my = sh_key + threadIdx.x * kPad;
+    int nv;  // how many of this thread's P blocks exist
+    {
+        K key[P];
+        unsigned valid;
+        load_keys<S>(score, B, first, key, valid);
+        nv = __popc(valid);  // the valid ones come first
+#pragma unroll
+        for (int j = 0; j < P; ++j) my[j] = key[j];
+    }
+    for (int i = threadIdx.x; i < kHistBins; i += kSelThreads) sh_hist[i] = 0;
+    if (threadIdx.x == 0) {
+        sh_boundary = -1;
+        sh_boundary_take = 0;
+    }
+    __syncthreads();
+    SEL_STAMP(st, 1);  // keys loaded
+    bool alive = true;
+
+    // ---- digit passes: tau = the k-th largest key, need = how many keys equal to tau are taken
+    u64 prefix = 0;
+    unsigned need = k;
+    if (!none) {
+        for (int p = 0; p < KT::kPasses && alive; ++p) {
+            const int shift = KT::shift(p), width = KT::width(p);
+            const u64 mask = (1ull << width) - 1;
+            if (KT::kSkippable && ((key_or >> shift) & mask) == 0) {  // this digit is 0 in every key
+                prefix <<= width;
+                continue;
+            }
+#pragma unroll 2
+            for (int j = 0; j < nv; ++j) {
+                const u64 key = my[j];
+                if (p == 0 || (key >> (shift + width)) == prefix) atomicAdd(&sh_hist[(unsigned)((key >> shift) & mask)], 1u);
+            }
+            __syncthreads();
+            SEL_STAMP(st, 2 + 4 * p);  // pass p: shared histogram built
+            for (int i = threadIdx.x; i < (1 << width); i += kSelThreads) {
+                const unsigned c = sh_hist[i];
+                if (c) {
+                    atomicAdd(&st->hist[p][i], c);
+                    sh_hist[i] = 0;  // ready for the next pass
+                }
+            }
+            SEL_STAMP(st, 3 + 4 * p);  // flushed
+            alive = sel_arrive_wait(&st->arrive[p], gridDim.x + never, st, info, &sh_ok);
+            SEL_STAMP(st, 4 + 4 * p);  // every CTA has arrived
+            if (alive) {
+                const unsigned d = width == 11 ? resolve_digit32_w<11>(st->hist[p], need, sh_scan, sh_out)
+                                               : resolve_digit32_w<10>(st->hist[p], need, sh_scan, sh_out);
+                prefix = (prefix << width) | d;
+            }
+            SEL_STAMP(st, 5 + 4 * p);  // digit resolved
+        }
+    }
+    const K tau = (K)prefix;
+
+    // ---- this CTA's record
+    unsigned gt_bits = 0, eq_bits = 0, my_gt = 0, my_eq = 0;
+    if (alive) {
+        unsigned c_nf = 0;
+#pragma unroll 2
+        for (int j = 0; j < nv; ++j) {
+            const K key = my[j];
+            if (SK::nonfinite(key)) ++c_nf;
+            if (none) continue;
+            if (key > tau) gt_bits |= 1u << j;
+            else if (key == tau) eq_bits |= 1u << j;
+        }
+        // per warp at most 256 of each: three 10-bit fields in one word, one warp-reduce instruction
+        const unsigned packed = __reduce_add_sync(0xffffffffu, __popc(gt_bits) | (__popc(eq_bits) << 10) | (c_nf << 20));
+        u64 lgt = 0, leq = 0;
+        if (!ulen) {
+            BlockLens bl(g, first);
+            for (int j = 0; j < nv; ++j) {
+                const u64 len = bl.next();
+                if (gt_bits >> j & 1u) lgt += len;
+                else if (eq_bits >> j & 1u) leq += len;
+            }
+            lgt = group_sum<32, u64>(lgt);
+            leq = group_sum<32, u64>(leq);
+        }
+        if ((threadIdx.x & 31) == 0) {
+            sh_w[threadIdx.x >> 5] = packed;
+            sh_wl[2 * (threadIdx.x >> 5)] = lgt;
+            sh_wl[2 * (threadIdx.x >> 5) + 1] = leq;
+        }
+        __syncthreads();
+        unsigned c_gt = 0, c_eq = 0, t_nf = 0;
+        lgt = leq = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const unsigned v = sh_w[w];
+            c_gt += v & 1023u, c_eq += (v >> 10) & 1023u, t_nf += v >> 20;
+        }
+        if (!ulen)
+            for (int w = 0; w < kWarps; ++w) lgt += sh_wl[2 * w], leq += sh_wl[2 * w + 1];
+        my_gt = c_gt, my_eq = c_eq;
+        SEL_STAMP(st, 26);  // own counts known
+        if (threadIdx.x == 0) {
+            SelRecord *r = &st->rec[blockIdx.x];
+            r->c_gt = c_gt;
+            r->c_eq = c_eq;
+            r->c_nf = t_nf;
+            r->len_gt = lgt;
+            r->len_eq = leq;
+            __threadfence();
+            st_release(&r->ready, 1u);
+        }
     }
 
-    // ---- the CTA that leaves last puts the shared state back for the next selection
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        sh_last = atomicAdd(&st->departed, 1u) == gridDim.x - 1;
-    }
-    __syncthreads();
-    if (!sh_last) return;
-    __threadfence();
-    for (int p = 0; p < KT::kPasses; ++p)
-        for (int i = threadIdx.x; i < kHistBins; i += kThreads) st->hist[p][i] = 0;
-    if (threadIdx.x == 0) {
-        const unsigned err = *reinterpret_cast<volatile unsigned *>(&st->error);
-        info->error = err;
-        if (err) {  // a barrier gave up: nothing was selected, and the pack kernel must copy nothing
-            info->k = 0;
-            info->payload_elems = 0;
+    // ---- exchange: thread c takes the record of CTA c; one packed scan gives every prefix sum
+    unsigned my_eq_before = 0, my_sel_base = 0, total_n = 0, total_nf = 0;
+    u64 my_len_base = 0, total_l = 0;
+    int cb = -1;
+    if (alive) {
+        const unsigned c = threadIdx.x;
+        unsigned e = 0, gt = 0, nf = 0;
+        u64 lg = 0, le = 0;
+        bool ok = true;
+        if (c < gridDim.x + never) {
+            const SelRecord *r = &st->rec[c];
+            ok = spin_until_at_least(&r->ready, 1u, st);
+            if (!ok) {
+                sel_fail(st, info);
+            } else if (c < gridDim.x) {
+                const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(r));
+                gt = v.x, e = v.y, nf = v.z;
+                if (!ulen) {
+                    lg = __ldcg(&r->len_gt);
+                    le = __ldcg(&r->len_eq);
+                }
+            }
         }
-        st->key_or = 0;  // forget which uint64 key bits were seen
-        st->barrier = 0;
-        st->departed = 0;
-        st->error = 0;
+        alive = __syncthreads_and(ok) != 0;
+        SEL_STAMP(st, 27);  // every CTA's record read
+        if (alive) {
+            // fewer than 2^21 keys in the whole grid (one tile of 4096 per CTA, fewer than 512 CTAs): three
+            // 21-bit fields
+            u64 tot;
+            const u64 ex = cta_excl_scan<u64, kSelThreads>((u64)gt | ((u64)e << 21) | ((u64)nf << 42), sh_scan64, &tot);
+            const unsigned ex_gt = (unsigned)(ex & 0x1fffffu), ex_e = (unsigned)((ex >> 21) & 0x1fffffu);
+            const unsigned tot_gt = (unsigned)(tot & 0x1fffffu), tot_e = (unsigned)((tot >> 21) & 0x1fffffu);
+            total_nf = (unsigned)(tot >> 42);
+            // the keys equal to tau are taken in id order, so the CTAs before c take min(need, ex_e) of them
+            const unsigned taken_before = need < ex_e ? need : ex_e;
+            unsigned take = need - taken_before;
+            if (take > e) take = e;
+            if (take != 0 && take != e) {  // the tau-keys run out inside CTA c's range
+                sh_boundary = (int)c;
+                sh_boundary_take = take;
+            }
+            total_n = tot_gt + (need < tot_e ? need : tot_e);
+            if (c == blockIdx.x) {
+                sh_mine[0] = ex_e;
+                sh_mine[1] = ex_gt + taken_before;
+            }
+            if (!ulen) {
+                const u64 l = lg + (take == e ? le : 0);
+                u64 two[2] = {c < blockIdx.x ? l : 0, l};
+                cta_sum_n<2, kSelThreads>(two, sh_wl);
+                my_len_base = two[0], total_l = two[1];
+            } else {
+                __syncthreads();
+            }
+            my_eq_before = (unsigned)sh_mine[0];
+            my_sel_base = (unsigned)sh_mine[1];
+            cb = sh_boundary;
+            if (ulen) {
+                my_len_base = (u64)my_sel_base * ulen;
+                total_l = (u64)total_n * ulen;
+            }
+        }
+    }
+
+    // ---- boundary: with blocks of different lengths, the CTAs behind the one where the tau-keys run out need
+    // the length of what it takes
+    if (alive && !ulen && cb >= 0 && (int)blockIdx.x >= cb) {
+        u64 *scan2 = sh_wl;  // free again
+        const u64 pl = boundary_len<S>(score, g, (unsigned)cb, 1u, gridDim.x, tau, sh_boundary_take, sh_scan64, scan2);
+        total_l += pl;
+        if ((int)blockIdx.x > cb) my_len_base += pl;
+    }
+    SEL_STAMP(st, 28);  // bases known
+
+    // ---- emit: ordered compaction of this CTA's tile
+    if (alive && !none) {
+        unsigned my_take = need > my_eq_before ? need - my_eq_before : 0;
+        if (my_take > my_eq) my_take = my_eq;
+        unsigned take_bits = gt_bits;
+        if (my_take == my_eq) {
+            take_bits |= eq_bits;
+        } else if (my_take != 0) {  // only in the CTA where the tau-keys run out (the same decision in all its threads)
+            unsigned rank = cta_excl_scan<unsigned, kSelThreads>(__popc(eq_bits), sh_scan, nullptr);
+            for (int j = 0; j < nv; ++j)
+                if (eq_bits >> j & 1u) {
+                    if (rank < my_take) take_bits |= 1u << j;
+                    ++rank;
+                }
+        }
+        if (ulen) {
+            unsigned pos = my_sel_base + cta_excl_scan<unsigned, kSelThreads>(__popc(take_bits), sh_scan, nullptr);
+            for (int j = 0; j < nv; ++j)
+                if (take_bits >> j & 1u) {
+                    sel[pos] = first + j;
+                    poff[pos] = (u64)pos * ulen;
+                    ++pos;
+                }
+        } else {
+            u64 lsum = 0;
+            BlockLens bl(g, first);
+            for (int j = 0; j < nv; ++j) {
+                const u64 len = bl.next();
+                if (take_bits >> j & 1u) lsum += len;
+            }
+            // one scan for both outputs: block counts in the top 16 bits (at most 4096 per tile), summed
+            // lengths below (a buffer has fewer than 2^48 elements: init rejects more)
+            const u64 both = cta_excl_scan<u64, kSelThreads>(((u64)__popc(take_bits) << 48) | lsum, sh_scan64, nullptr);
+            unsigned pos = my_sel_base + (unsigned)(both >> 48);
+            u64 off = my_len_base + (both & ((1ull << 48) - 1));
+            BlockLens bl2(g, first);
+            for (int j = 0; j < nv; ++j) {
+                const u64 len = bl2.next();
+                if (take_bits >> j & 1u) {
+                    sel[pos] = first + j;
+                    poff[pos] = off;
+                    ++pos;
+                    off += len;
+                }
+            }
+        }
+    }
+    SEL_STAMP(st, 29);  // emitted
+    // The last CTA lies behind every boundary, so its totals are complete.  By now every CTA has read key_or.
+    if (alive && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {
+        info->k = total_n;
+        info->payload_elems = total_l;
+        info->nonfinite_blocks = total_nf;
+        poff[total_n] = total_l;
+        if (KT::kSkippable) st->key_or = 0;  // forget which uint64 key bits were seen
     }
 }
 

@@ -233,6 +233,31 @@ def test_few_distinct_scores_many_ties():
         ck.close()
 
 
+@pytest.mark.parametrize("kind", ["f32", "i32"])
+def test_more_blocks_than_one_selection_tile_per_cta(kind):
+    """Beyond 4096 blocks per SM the selection's CTAs walk several tiles each and re-read their keys (another
+    kernel than the one-tile-per-CTA form): 700 000 blocks of 4 elements, many exact ties at zero, and a k that
+    ends inside the ties."""
+    r = rng(21)
+    nb, blk = 700_000, 4
+    geom = Geometry(nb * blk, 0, blk, 8)
+    if kind == "f32":
+        z = r.standard_normal(nb * blk).astype(np.float32)
+        d = r.standard_normal(nb * blk).astype(np.float32) * np.repeat(r.lognormal(0, 1, nb), blk).astype(np.float32)
+    else:
+        z = r.integers(0, 50, size=nb * blk).astype(np.int32)
+        d = r.integers(-3, 4, size=nb * blk).astype(np.int32)
+    d.reshape(nb, blk)[r.random(nb) < 0.5] = 0  # half of the blocks unchanged: score exactly 0
+    x = (z + d).astype(z.dtype)
+    boff = block_offsets(geom)
+    for k in (1, 70_001, 350_000 + 12_345, nb - 3):
+        xd = parity.to_dev(x)
+        ck = parity.make_ctx(xd, z, geom=geom)
+        ora = oracle.priority_save(x, z, boff, k=k)
+        parity.check_save(ck, ck.priority_save_k(k), x, z, boff, ora)
+        ck.close()
+
+
 def test_uint64_keys_above_32_bits():
     r = rng(8)
     nb, blk = 4000, 16
@@ -418,9 +443,9 @@ def test_launch_count_profile_and_last_info():
     ms = api.scar_ckpt_profile_read(ck.ctx)
     assert ms[0] > 0 and ms[1] > 0 and ms[2] > 0 and ms[3] == 0 and ms[4] == 0
     ck.recover_partial(w.lost_shards, sync=False)
-    assert api.scar_ckpt_launch_count(ck.ctx) - n1 == 2
+    assert api.scar_ckpt_launch_count(ck.ctx) - n1 == 1  # restore and norm reduction are one kernel
     ms = api.scar_ckpt_profile_read(ck.ctx)
-    assert ms[3] > 0 and ms[4] > 0 and ms[0] == 0
+    assert ms[3] > 0 and ms[4] >= 0 and ms[0] == 0
     s, nrm = api.scar_ckpt_last_info(ck.ctx)
     assert int(s.k) == 64 and int(nrm.lost_blocks) == 128
     ck.block_scores()

@@ -85,9 +85,11 @@ def test_stored_checkpoint_with_explicit_offsets_and_io_errors(tmp_path):
     ck = parity.make_ctx(xd, z, boff=boff, n_shards=1)
     ck.store_full(fd)
     assert file_bytes(path) == z.tobytes()
-    ck.drain_init(nb, int(boff[-1]))
-    with pytest.raises(api.ScarError):
-        ck.priority_save_k(2)  # 2 x (longest block) exceeds the slot: the capacity rule is per block count
+    lens = np.sort(np.diff(boff.astype(np.int64)))[::-1]
+    ck.drain_init(nb, int(lens[0] + lens[1] - 1))
+    with pytest.raises(api.ScarError) as e:
+        ck.priority_save_k(2)  # the capacity rule: the k longest blocks of the layout must fit the slot
+    assert e.value.code == -7
     ora = oracle.priority_save(x, z, boff, k=1)
     parity.check_save(ck, ck.priority_save_k(1), x, z, boff, ora)
     t = ck.drain_enqueue()

@@ -701,3 +701,40 @@ def test_workload_recipes_have_the_stated_structure():
     assert oracle.block_scores(wl.x, wl.z, block_offsets(wl.geom)).dtype == np.uint64
     wm = make_workload("mf", l_rows=960, r_rows=36, seed=2)
     assert wm.lost_blocks.sum() == 240 and wm.lost_blocks[960:].sum() == 0
+
+
+# ------------------------------------------------------------------ the OpenMP build (timing only)
+
+
+def test_openmp_build_of_the_oracle_agrees_with_the_plain_build():
+    """The all-core CPU baseline times the same source compiled with -fopenmp.  Integer results, ids, payload
+    bytes and restored buffers must be bit-identical to the plain build's, per-block float scores too (each block
+    is still summed in element order by one thread); only the recovery's sum across blocks changes its order."""
+    import oracle as ora
+
+    r = np.random.Generator(np.random.PCG64(77))
+    nb = 3000
+    lens = r.integers(0, 200, size=nb)
+    boff = np.concatenate([[0], np.cumsum(lens)]).astype(np.uint64)
+    n = int(boff[-1])
+    lost = (r.random(nb) < 0.4).astype(np.uint8)
+    cases = []
+    zf = r.standard_normal(n).astype(np.float32)
+    cases.append((zf + r.standard_normal(n).astype(np.float32) * np.float32(0.1), zf))
+    zi = r.integers(-1000, 1000, size=n).astype(np.int32)
+    cases.append(((zi + r.integers(-5, 6, size=n)).astype(np.int32), zi))
+    got = {}
+    try:
+        for omp in (False, True):
+            threads = ora.use_openmp(omp)
+            assert threads >= 1 and (omp or threads == 1)
+            got[omp] = [(ora.priority_save(x, z, boff, k=700), ora.perturbation_norm(x, z, boff, lost),
+                         ora.recover_partial(x, z, boff, lost)) for x, z in cases]
+    finally:
+        ora.use_openmp(False)
+    for (s0, n0, (r0, x0)), (s1, n1, (r1, x1)) in zip(got[False], got[True]):
+        assert s0.scores.tobytes() == s1.scores.tobytes() and s0.sel.tobytes() == s1.sel.tobytes()
+        assert s0.payload.tobytes() == s1.payload.tobytes() and s0.poff.tobytes() == s1.poff.tobytes()
+        assert s0.z_after.tobytes() == s1.z_after.tobytes() and x0.tobytes() == x1.tobytes()
+        assert (n0.l1, n0.lost_blocks, n0.lost_elems) == (n1.l1, n1.lost_blocks, n1.lost_elems)
+        assert abs(n0.sumsq - n1.sumsq) <= 1e-13 * max(n0.sumsq, 1e-300) and abs(r0.l2 - r1.l2) <= 1e-13 * max(r0.l2, 1e-300)
