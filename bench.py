@@ -71,10 +71,10 @@ def recorded_traffic(n_elems: int, kernel: str = "k_block_scores"):
 
     pkg = os.path.join(ROOT, "paper_1810_07354_b200")
     try:
-        with open(os.path.join(pkg, "ncu_traffic.json")) as f:
+        with open(os.path.join(ROOT, "profiles", "ncu_traffic.json")) as f:
             rec = json.load(f)[kernel]
         h = hashlib.sha256()
-        for name in ("geom.cuh", "block_pass.cuh"):
+        for name in ("geom.cuh", "sel_state.cuh", "block_pass.cuh"):
             with open(os.path.join(pkg, "csrc", name), "rb") as f:
                 h.update(f.read())
         if h.hexdigest() != rec["src_sha256"]:
@@ -550,6 +550,120 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_sharded(args):
+    """The multi-GPU form of the save (Section 4.3 with one GPU per node): the CNN-scale parameter vector is
+    split over the ranks by blocks, every rank scores its slice, one all-gather makes all scores known, every
+    rank selects the same global fraction and saves the blocks it owns.  Total work is fixed as N grows
+    ("scaling": "strong").  A step = one sharded save per r of the sweep + the rank's full norm + a recovery of
+    one of its 8 local shards; device-timed per call, maximum over ranks."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_1810_07354_b200 import api
+    from paper_1810_07354_b200.sharded import ShardedCheckpoint, rank_block_range
+    from workloads.configs import make_cnn_device
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback for the library")
+    api.load_library()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    nb_global = args.n_elems // BLOCK
+    lo, hi = rank_block_range(nb_global, world, rank)
+    n = (hi - lo) * BLOCK
+    _, z0, x0, lost_shards = make_cnn_device(n, BLOCK, seed=4 + rank, device=dev)
+    x = x0.clone()
+    sc = ShardedCheckpoint(x, nb_global, world, rank, n_shards=8, block_elems=BLOCK)
+    z_lib = sc.ck.views()["z"]
+    flush = torch.empty(64 << 20, dtype=torch.float32, device=dev)
+    r_sweep = (0.01, 0.1, 0.5, 1.0)
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+
+    def one_step(rec):
+        for r in r_sweep:
+            z_lib.copy_(z0)
+            flush.zero_()
+            barrier()  # the exchange inside the save would otherwise absorb the ranks' skew
+            a, b = ev(), ev()
+            a.record()
+            sc.priority_save(r=r)
+            b.record()
+            rec.append((("save", r), a, b))
+        z_lib.copy_(z0)
+        flush.zero_()
+        a, b = ev(), ev()
+        a.record()
+        sc.ck.perturbation_norm(None, sync=False)
+        b.record()
+        rec.append((("norm", None), a, b))
+        flush.zero_()
+        a, b = ev(), ev()
+        a.record()
+        sc.ck.recover_partial(lost_shards, sync=False)
+        b.record()
+        rec.append((("recover", None), a, b))
+        x.copy_(x0)
+
+    for _ in range(args.warmup):
+        one_step([])
+    barrier()
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid)) if rank == 0 else None
+    launches0 = api.scar_ckpt_launch_count(sc.ck.ctx)
+    rec = []
+    barrier()
+    w0 = time.time()
+    for _ in range(args.steps):
+        one_step(rec)
+    barrier()
+    w1 = time.time()
+    launches = api.scar_ckpt_launch_count(sc.ck.ctx) - launches0
+    clocks = sampler.stop(w0, w1) if sampler else None
+    t = {}
+    for key, a, b in rec:
+        t.setdefault(key, []).append(a.elapsed_time(b))
+    keys = sorted(t, key=str)
+    sums = max_over_ranks([sum(t[k]) for k in keys], dev, world)
+    tot = dict(zip(keys, sums))
+    if rank == 0:
+        save_ms = sum(v for (kind, _), v in tot.items() if kind == "save")
+        tot_ms = sum(tot.values())
+        scanned = 2 * nb_global * BLOCK * ELEM
+        peak, peak_kind = hbm_peak()
+        line = {
+            "metric": METRIC, "value": len(r_sweep) * scanned * args.steps / (save_ms * 1e-3) / 1e9, "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot_ms / args.steps,
+            "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": DESCRIPTIONS["cnn"] + " [blocks split over the ranks, global top-r]",
+                       "n_elems": nb_global * BLOCK, "n_blocks": nb_global, "r_sweep": list(r_sweep),
+                       "parallelism": f"blocks sharded x{world}, one all-gather of the scores per save",
+                       "l2": "per-rank inputs larger than L2 up to 8 ranks; L2 flushed before every timed call"},
+            "per_r": {str(r): {"save_ms": tot[("save", r)] / args.steps,
+                               "scanned_gbs": scanned / (tot[("save", r)] / args.steps) / 1e6} for r in r_sweep},
+            "perturbation_norm_ms": tot[("norm", None)] / args.steps,
+            "partial_recovery_ms": tot[("recover", None)] / args.steps,
+            "roofline": {"bound": "hbm", "kernel": "k_block_scores", "achieved": None, "peak": peak, "unit": "GB/s",
+                         "frac": None, "peak_source": f"of {peak_kind}", "traffic": None,
+                         "note": "per-kernel figures are those of the single-GPU line; this mode times whole calls"},
+            "gpu_launches": int(launches), "clocks": clocks, "wall_s_timed_region": w1 - w0,
+        }
+        print(json.dumps(line))
+    barrier()
+    sc.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def run_extras(api, ck, x, x0, z_lib, z0, geom, r_sweep, flush, dev, with_bylayer):
     """Measurements beside the headline step, outside its timed region: the two baseline selectors
     (Section 5.4), the asynchronous drain (Section 4.3) and a by-layer layout with very unequal blocks
@@ -712,6 +826,9 @@ def main():
     ap.add_argument("--workload", default="cnn", choices=sorted(DESCRIPTIONS))
     ap.add_argument("--n-elems", type=int, default=N_ELEMS,
                     help="elements of the CNN-scale parameter vector (default 2**30)")
+    ap.add_argument("--sharded", action="store_true",
+                    help="multi-GPU form of the save: the blocks of one parameter vector split over the ranks, "
+                         "global top-r through one all-gather of the scores (strong scaling) instead of replicas")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true",
@@ -721,6 +838,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.sharded:
+        run_sharded(args)
     else:
         run_gpu(args)
 

@@ -24,9 +24,13 @@
  *   - All GPU work of a context runs on the CUDA stream given at init, in call
  *     order.  A call whose result pointer `out` is NULL only enqueues; with a
  *     non-NULL `out` it also waits for the stream and fills `out`.
- *     Enqueue-only calls use no host synchronisation and can be recorded by
- *     CUDA stream capture on the context's stream (saves, recoveries with
- *     shard masks or device block masks, norms, scar_ckpt_load).
+ *     Enqueue-only calls use no host synchronisation and read no caller-owned
+ *     host memory after they return, so they can be recorded by CUDA stream
+ *     capture on the context's stream: saves, recoveries and norms with device
+ *     block masks or with shard masks of up to 1024 shards (their flags travel
+ *     in launch parameters; a replay uses the mask of the capture), and
+ *     scar_ckpt_load.  A shard-mask call on a context with more than 1024
+ *     shards waits for the stream and is not capturable.
  *   - One context serves one caller at a time (no internal locking).
  *   - There is no CPU fallback: without a usable CUDA device init fails.
  */
@@ -61,8 +65,8 @@ enum {
     SCAR_ERR_ALLOC = -3,       /* device or host allocation failed */
     SCAR_ERR_CUDA = -4,        /* a CUDA runtime call or kernel launch failed */
     SCAR_ERR_STATE = -5,       /* call not valid in the context's current state */
-    SCAR_ERR_TIMEOUT = -6,     /* a bounded device-side wait (grid barrier of the selection) gave up;
-                                  the save's outputs are invalid, the context stays usable */
+    SCAR_ERR_TIMEOUT = -6,     /* a bounded device-side wait (of the selection, or of the norm reduction) gave
+                                  up; the call's outputs are invalid, the context stays usable */
     SCAR_ERR_CAPACITY = -7,    /* problem larger than a fixed-size internal buffer */
     SCAR_ERR_IO = -8           /* a read or write of the stored checkpoint failed or came up short */
 };
@@ -135,8 +139,43 @@ int scar_ckpt_block_scores(scar_ctx *ctx);
  * traditional full checkpoint.  r outside [0,1] or NaN: SCAR_ERR_INVALID_ARG. */
 int scar_ckpt_priority_save(scar_ctx *ctx, double r, scar_save_info *out);
 
+/* The rule that turns the fraction r of Section 4.2 into a block count, as
+ * scar_ckpt_priority_save applies it: k = round(r * n_blocks), halves away from
+ * zero, at least 1 when r > 0 and n_blocks > 0, at most n_blocks.  For callers
+ * that schedule saves themselves (the baseline selectors take k, not r).  Host
+ * only.  SCAR_ERR_INVALID_ARG for r outside [0,1], NaN, or k == NULL. */
+int scar_k_from_r(double r, uint64_t n_blocks, uint64_t *k);
+
 /* Same with the block count given directly (0 <= k <= B). */
 int scar_ckpt_priority_save_k(scar_ctx *ctx, uint64_t k, scar_save_info *out);
+
+/* The multi-GPU form of a prioritized save: the checkpoint protocol of Section
+ * 4.3 the way the paper runs it, with one GPU per parameter-server node.  Every
+ * node scores its own partition (step 1: scar_ckpt_block_scores), the scores of
+ * all nodes are made known to all (step 2: the caller's exchange, e.g. an NCCL
+ * all-gather of the score arrays; the library itself has no communication), and
+ * every node selects the same global fraction and saves what it owns (steps 3
+ * and 4: this call).  Payloads never leave their GPU; recovery stays a local
+ * call on whichever context owns the lost blocks.
+ *
+ * The context covers this rank's partition: its B blocks are blocks
+ * [first_block, first_block + B) of a global layout of n_global_blocks blocks.
+ *   d_global_scores  DEVICE array of n_global_blocks scores in global block
+ *                    order, of the context's score type (float32 / uint64), as
+ *                    scar_ckpt_view returns them per rank; read when the
+ *                    enqueued work runs
+ *   k_global         blocks to save over all ranks (e.g. scar_k_from_r(r,
+ *                    n_global_blocks)), 0 <= k_global <= n_global_blocks
+ * The k_global highest global scores are selected, ties to the lowest global
+ * id; the ones in this rank's range are packed and refreshed exactly as by a
+ * single-GPU save: sel holds LOCAL block ids, ascending, out->k is this rank's
+ * count, out->nonfinite_blocks counts over all ranks.  The union over ranks of
+ * the saved blocks (local id + first_block) is what one context over the
+ * concatenated buffer would have saved.  Always waits for the stream (the
+ * rank's count crosses to the host once), so `out` must not be NULL and the
+ * call cannot be captured. */
+int scar_ckpt_priority_save_sharded(scar_ctx *ctx, const void *d_global_scores, uint64_t n_global_blocks,
+                                    uint64_t first_block, uint64_t k_global, scar_save_info *out);
 
 /* The two baseline selectors the paper compares the prioritized checkpoint with
  * (Section 5.4).  Both skip the scoring pass (the score array keeps the values
@@ -185,10 +224,10 @@ int scar_perturbation_norm_blocks(scar_ctx *ctx, const uint8_t *d_lost_blocks, s
  * that cannot take the device-wide synchronisation an allocation implies, or a
  * plug-in whose host forbids it to grow its memory.  This call needs no
  * context and calls no cudaMalloc / cudaFree or other allocating routine.  Its
- * per-block partial sums live in a fixed array of about 8 MiB inside the
- * library's device image (every GPU that loads the library holds it until the
- * process exits), which caps the problem at SCAR_STATIC_MAX_BLOCKS blocks;
- * larger layouts return SCAR_ERR_CAPACITY and nothing is enqueued.
+ * partial sums live in a fixed array of about 0.4 MiB inside the library's
+ * device image (every GPU that loads the library holds it until the process
+ * exits), which caps the problem at SCAR_STATIC_MAX_BLOCKS blocks; larger
+ * layouts return SCAR_ERR_CAPACITY and nothing is enqueued.
  *
  *   d_x, d_z       DEVICE buffers of layout->n_elems elements of type dt, both
  *                  16-byte aligned, read only; z is the checkpoint to compare with
@@ -198,10 +237,15 @@ int scar_perturbation_norm_blocks(scar_ctx *ctx, const uint8_t *d_lost_blocks, s
  *   cuda_stream    cudaStream_t to enqueue on; the call does not wait
  *
  * The first call on each device looks up the array's device address (once, with
- * that device current); make that first call before any stream capture.  All
- * calls on a device share the one array: calls whose GPU work overlaps (different
- * streams, or different threads) race and give wrong results; calls ordered on
- * one stream are fine.  Results are bit-identical to scar_perturbation_norm_blocks. */
+ * that device current), and with CUDA's lazy module loading it is also what
+ * brings the array and this call's kernels onto the device, which itself needs
+ * a little device memory.  So make the first call at start-up, before memory
+ * can run short and before any stream capture: a call with n_elems == 0 does the
+ * look-up, one tiny real call loads the kernels.  All calls on a device share
+ * the one array (each call first empties the part it uses): calls whose GPU
+ * work overlaps (different streams, or different threads) race and give wrong
+ * results; calls ordered on one stream are fine.  Results are bit-identical to
+ * scar_perturbation_norm_blocks. */
 #define SCAR_STATIC_MAX_BLOCKS (1ull << 20)
 int scar_perturbation_norm_static(const void *d_x, const void *d_z, scar_dtype dt, const scar_layout *layout,
                                   const uint8_t *d_lost_blocks, scar_norm_info *d_out, void *cuda_stream);
@@ -308,8 +352,9 @@ uint64_t scar_ckpt_launch_count(const scar_ctx *ctx);
  * its phases with CUDA events on the context's stream.  phase_ms receives the
  * duration of the most recent call's phases, in milliseconds, after waiting for
  * the stream: [0] block scores, [1] selection, [2] pack + cache refresh,
- * [3] restore / norm pass, [4] final reduction; phases a call did not run
- * read 0. */
+ * [3] restore / norm pass including its reduction (one kernel), [4] the
+ * reduction as a kernel of its own (layouts cut into segments only, else 0);
+ * phases a call did not run read 0. */
 int scar_ckpt_profile(scar_ctx *ctx, int enable);
 int scar_ckpt_profile_read(scar_ctx *ctx, float phase_ms[5]);
 
@@ -335,14 +380,14 @@ double scar_iteration_cost_bound(double delta_T, double dist0, double c);
 double scar_irreducible_error(double delta_max, double c);
 
 /* Self-test hook for the bounded device-side wait.  The selection kernel's
- * CTAs meet at grid barriers whose wait gives up after a fixed number of tries
- * instead of hanging.  This call mis-sets the barrier's arrival counter (nothing
- * else), so that the first barrier of the NEXT prioritized or random save can
- * never complete: that save takes about a second (the length of the bounded
- * wait), selects and copies nothing, leaves z untouched, and returns
- * SCAR_ERR_TIMEOUT from the call that reads its result (the save itself with a
- * non-NULL out, or scar_ckpt_last_info).  The kernel puts the barrier state back
- * on its way out, so the save after that one works normally.  Enqueue only.
+ * CTAs meet at a few points whose wait gives up after a fixed number of polls
+ * (2^20: a quarter of a second at the earliest, about a second in practice)
+ * instead of hanging.  This call makes the NEXT prioritized or random save
+ * expect one arrival more than its selection has CTAs (host state only), so
+ * that its first wait can never complete: that save takes about a second,
+ * selects and copies nothing, leaves z untouched, and returns SCAR_ERR_TIMEOUT
+ * from the call that reads its result (the save itself with a non-NULL out, or
+ * scar_ckpt_last_info).  The save after that one works normally.
  * SCAR_ERR_STATE on an empty buffer. */
 int scar_ckpt_selftest_arm_timeout(scar_ctx *ctx);
 

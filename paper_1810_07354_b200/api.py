@@ -65,7 +65,9 @@ _SIGS = {
     "scar_ckpt_set_norm": (_int, [_vp, _int, _vp]),
     "scar_ckpt_block_scores": (_int, [_vp]),
     "scar_ckpt_priority_save": (_int, [_vp, _dbl, C.POINTER(scar_save_info)]),
+    "scar_k_from_r": (_int, [_dbl, _u64, C.POINTER(_u64)]),
     "scar_ckpt_priority_save_k": (_int, [_vp, _u64, C.POINTER(scar_save_info)]),
+    "scar_ckpt_priority_save_sharded": (_int, [_vp, _vp, _u64, _u64, _u64, C.POINTER(scar_save_info)]),
     "scar_ckpt_save_round": (_int, [_vp, _u64, C.POINTER(scar_save_info)]),
     "scar_ckpt_save_random": (_int, [_vp, _u64, _vp, C.POINTER(scar_save_info)]),
     "scar_ckpt_round_cursor": (_int, [_vp, C.POINTER(_u64), C.POINTER(_u64)]),
@@ -181,10 +183,25 @@ def scar_ckpt_priority_save(ctx: int, r: float, sync: bool = True) -> Optional[s
     return out
 
 
+def scar_k_from_r(r: float, n_blocks: int) -> int:
+    """The library's rule for the number of blocks a fraction r stands for."""
+    k = _u64(0)
+    _check(load_library().scar_k_from_r(r, n_blocks, C.byref(k)), "scar_k_from_r")
+    return int(k.value)
+
+
 def scar_ckpt_priority_save_k(ctx: int, k: int, sync: bool = True) -> Optional[scar_save_info]:
     out = _save_out(sync)
     _check(load_library().scar_ckpt_priority_save_k(ctx, k, C.byref(out) if sync else None),
            "scar_ckpt_priority_save_k")
+    return out
+
+
+def scar_ckpt_priority_save_sharded(ctx: int, d_global_scores, n_global_blocks: int, first_block: int,
+                                    k_global: int) -> scar_save_info:
+    out = scar_save_info()
+    _check(load_library().scar_ckpt_priority_save_sharded(ctx, _addr(d_global_scores), n_global_blocks, first_block,
+                                                          k_global, C.byref(out)), "scar_ckpt_priority_save_sharded")
     return out
 
 
@@ -444,6 +461,9 @@ class ScarCheckpoint:
 
     def priority_save_k(self, k: int, sync: bool = True):
         return scar_ckpt_priority_save_k(self.ctx, k, sync)
+
+    def priority_save_sharded(self, d_global_scores, n_global_blocks: int, first_block: int, k_global: int):
+        return scar_ckpt_priority_save_sharded(self.ctx, d_global_scores, n_global_blocks, first_block, k_global)
 
     def save_round(self, k: int, sync: bool = True):
         return scar_ckpt_save_round(self.ctx, k, sync)

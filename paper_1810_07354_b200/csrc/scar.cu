@@ -78,8 +78,12 @@ struct scar_ctx {
     uint8_t *h_shard_mask = nullptr;  // pinned staging copy of such a mask
     uint8_t *d_block_mask = nullptr;  // only used when a shard mask has too many runs
     SelState *st = nullptr;
-    unsigned n_sel_tiles = 0;
-    unsigned sel_grid = 1, sel_tiles_per_cta = 1;  // launch shape of the cooperative selection kernel
+    // multi-GPU form of a save (scar_ckpt_priority_save_sharded): scratch for the selection over all ranks' scores
+    OutSet glob{};                 // ids / offsets / record of the global selection (no payload)
+    uint64_t glob_blocks = 0;      // capacity of glob in blocks
+    uint32_t *member = nullptr;    // B flags: this rank's blocks that the global selection took
+    unsigned long long *d_count = nullptr;  // how many
+    unsigned long long *h_count = nullptr;  // pinned
     bool arm_never = false;  // self-test: the next selection's waits expect an arrival that never comes
     int n_sms = 1;
     NormScratch rs{};  // per-CTA / per-tile partials and tickets of the fused norm reduction
@@ -308,33 +312,53 @@ template <typename T, int NORM> void launch_full_save(scar_ctx *c) {
     ++c->launches;
 }
 
-// a2: one cooperative launch (all CTAs resident, so its waits cannot deadlock).  The selection state must be
-// zero when the kernel starts: the scoring pass that precedes a prioritized save clears it (pre_cleared), any
-// other caller gets a memset here.
-template <typename S> int launch_select(scar_ctx *c, const S *score, uint64_t k, bool pre_cleared) {
+// Launch shape of a selection over n_blocks keys: contiguous tile ranges over at most one CTA per SM (few enough
+// that a meeting of all CTAs costs a couple of microseconds, always resident, and fewer than the exchange has
+// threads).
+struct SelectShape {
+    unsigned n_tiles, tiles_per_cta, grid;
+};
+SelectShape select_shape(const scar_ctx *c, uint64_t n_blocks) {
+    SelectShape sh;
+    sh.n_tiles = (unsigned)((n_blocks + kSelTile - 1) / kSelTile);
+    if (sh.n_tiles == 0) sh.n_tiles = 1;
+    const unsigned cap = (unsigned)c->n_sms < (unsigned)kMaxSelCtas - 1 ? (unsigned)c->n_sms : (unsigned)kMaxSelCtas - 1;
+    sh.tiles_per_cta = (sh.n_tiles + cap - 1) / cap;
+    sh.grid = (sh.n_tiles + sh.tiles_per_cta - 1) / sh.tiles_per_cta;
+    return sh;
+}
+
+// a2: one cooperative launch (all CTAs resident, so its waits cannot deadlock) over the keys `score` of the
+// blocks of `g`, writing ids, offsets and the result record to `to`.  The selection state must be zero when the
+// kernel starts: the scoring pass that precedes a prioritized save clears it (pre_cleared), any other caller
+// gets a memset here.
+template <typename S>
+int launch_select(scar_ctx *c, const S *score, const Geom &g, uint64_t k, const OutSet &to, bool pre_cleared) {
     if (!pre_cleared) {
         CU_TRY(cudaMemsetAsync(reinterpret_cast<char *>(c->st) + kSelZeroFrom, 0, sizeof(SelState) - kSelZeroFrom,
                                c->stream));
-        CU_TRY(cudaMemsetAsync(c->cur.info, 0, sizeof(SaveInfoDev), c->stream));
+        CU_TRY(cudaMemsetAsync(to.info, 0, sizeof(SaveInfoDev), c->stream));
     }
+    const SelectShape sh = select_shape(c, g.n_blocks);
+    Geom geom = g;
+    OutSet out = to;
     unsigned long long kk = k;
-    unsigned k32 = (unsigned)k, nt = c->n_sel_tiles, per = c->sel_tiles_per_cta, never = c->arm_never ? 1u : 0u;
+    unsigned k32 = (unsigned)k, nt = sh.n_tiles, per = sh.tiles_per_cta, never = c->arm_never ? 1u : 0u;
     c->arm_never = false;
     if (per == 1) {  // the usual case: one tile per CTA
-        void *args[] = {&score, &c->g, &k32, &c->st, &c->cur.info, &c->cur.sel, &c->cur.poff, &never};
-        CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select_tile<S>), dim3(c->sel_grid),
+        void *args[] = {&score, &geom, &k32, &c->st, &out.info, &out.sel, &out.poff, &never};
+        CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select_tile<S>), dim3(sh.grid),
                                            dim3(kSelThreads), args, 0, c->stream));
     } else {
-        void *args[] = {&score, &c->g, &kk, &c->st, &c->cur.info, &c->cur.sel, &c->cur.poff, &nt, &per, &never};
-        CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select<S, false>), dim3(c->sel_grid),
+        void *args[] = {&score, &geom, &kk, &c->st, &out.info, &out.sel, &out.poff, &nt, &per, &never};
+        CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select<S, false>), dim3(sh.grid),
                                            dim3(kSelThreads), args, 0, c->stream));
     }
     ++c->launches;
     return SCAR_OK;
 }
 
-// Grid of the selection kernel: contiguous tile ranges over at most one CTA per SM (few enough that a meeting
-// of all CTAs costs a couple of microseconds, always resident, and fewer than the exchange has threads).
+// Checks once that the selection kernels can be launched cooperatively and notes the SM count.
 template <typename S> int select_occupancy(int &occ) {
     int o = 0;
     CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, k_select<S, false>, kSelThreads, 0));
@@ -353,10 +377,6 @@ int plan_select(scar_ctx *c) {
         return rc;
     if (!coop || sms < 1 || occ < 1) return SCAR_ERR_CUDA;
     c->n_sms = sms;
-    const unsigned cap = (unsigned)sms < (unsigned)kMaxSelCtas - 1 ? (unsigned)sms : (unsigned)kMaxSelCtas - 1;
-    const unsigned nt = c->n_sel_tiles;
-    c->sel_tiles_per_cta = (nt + cap - 1) / cap;
-    c->sel_grid = (nt + c->sel_tiles_per_cta - 1) / c->sel_tiles_per_cta;
     return SCAR_OK;
 }
 
@@ -579,8 +599,8 @@ int enqueue_save(scar_ctx *c, uint64_t k) {
     record(c, 1);
     const int rc_sel =
         c->dt == SCAR_F32
-            ? launch_select<float>(c, static_cast<const float *>(c->score), k, true)
-            : launch_select<unsigned long long>(c, static_cast<const unsigned long long *>(c->score), k, true);
+            ? launch_select<float>(c, static_cast<const float *>(c->score), c->g, k, c->cur, true)
+            : launch_select<unsigned long long>(c, static_cast<const unsigned long long *>(c->score), c->g, k, c->cur, true);
     if (rc_sel != SCAR_OK) {
         cudaGetLastError();
         return rc_sel;
@@ -611,7 +631,7 @@ int enqueue_baseline_save(scar_ctx *c, uint64_t k, const uint32_t *d_priorities)
         return SCAR_OK;
     }
     if (d_priorities) {
-        const int rc = launch_select<unsigned>(c, d_priorities, k, false);
+        const int rc = launch_select<unsigned>(c, d_priorities, c->g, k, c->cur, false);
         if (rc != SCAR_OK) {
             cudaGetLastError();
             return rc;
@@ -785,8 +805,6 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
 
     const uint64_t N = g.n_elems, B = g.n_blocks;
     const size_t score_bytes = (dt == SCAR_F32 ? 4 : 8) * B;
-    c->n_sel_tiles = (unsigned)((B + kSelTile - 1) / kSelTile);
-    if (c->n_sel_tiles == 0) c->n_sel_tiles = 1;
     const bool long_blocks = c->max_block_len > 2 * kSegElems;
 
     rc = SCAR_OK;
@@ -910,6 +928,11 @@ int scar_ckpt_block_scores(scar_ctx *c) {
     return SCAR_OK;
 }
 
+int scar_k_from_r(double r, uint64_t n_blocks, uint64_t *k) {
+    if (!k) return SCAR_ERR_INVALID_ARG;
+    return k_from_r(r, n_blocks, k);
+}
+
 int scar_ckpt_priority_save_k(scar_ctx *c, uint64_t k, scar_save_info *out) {
     if (!c || k > c->g.n_blocks) return SCAR_ERR_INVALID_ARG;
     int rc = check_device(c);
@@ -925,6 +948,87 @@ int scar_ckpt_priority_save(scar_ctx *c, double r, scar_save_info *out) {
     int rc = k_from_r(r, c->g.n_blocks, &k);
     if (rc != SCAR_OK) return rc;
     return scar_ckpt_priority_save_k(c, k, out);
+}
+
+int scar_ckpt_priority_save_sharded(scar_ctx *c, const void *d_global_scores, uint64_t n_global_blocks,
+                                    uint64_t first_block, uint64_t k_global, scar_save_info *out) {
+    if (!c || !out) return SCAR_ERR_INVALID_ARG;
+    const uint64_t B = c->g.n_blocks;
+    if (n_global_blocks > 0xfffffffeull || first_block > n_global_blocks || B > n_global_blocks - first_block ||
+        k_global > n_global_blocks || (!d_global_scores && n_global_blocks))
+        return SCAR_ERR_INVALID_ARG;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    if (n_global_blocks == 0 || B == 0) {  // nothing of this rank's to choose from: an empty save
+        if ((rc = enqueue_baseline_save(c, 0, nullptr)) != SCAR_OK) return rc;
+        return fetch_save(c, out);
+    }
+    // scratch for the selection over all ranks' scores, grown on demand
+    if (c->glob_blocks < n_global_blocks) {
+        CU_TRY(cudaStreamSynchronize(c->stream));
+        if (c->glob.sel) {  // the smaller buffers stay owned (and are freed at destroy); layouts rarely change size
+            c->glob = OutSet{};
+            c->glob_blocks = 0;
+        }
+        if ((rc = dev_alloc(c, &c->glob.sel, n_global_blocks * 4)) != SCAR_OK ||
+            (rc = dev_alloc(c, &c->glob.poff, (n_global_blocks + 1) * 8)) != SCAR_OK ||
+            (!c->glob.info && (rc = dev_alloc(c, &c->glob.info, sizeof(SaveInfoDev))) != SCAR_OK))
+            return rc;
+        c->glob_blocks = n_global_blocks;
+    }
+    if (!c->member) {
+        if ((rc = dev_alloc(c, &c->member, B * 4)) != SCAR_OK || (rc = dev_alloc(c, &c->d_count, 3 * 8)) != SCAR_OK)
+            return rc;
+        void *q = nullptr;
+        if (cudaMallocHost(&q, 3 * 8) != cudaSuccess) {
+            cudaGetLastError();
+            return SCAR_ERR_ALLOC;
+        }
+        c->owned_host.push_back(q);
+        c->h_count = static_cast<unsigned long long *>(q);
+    }
+    if ((rc = save_fits(c, B < k_global ? B : k_global)) != SCAR_OK) return rc;  // this rank saves at most min(B, k) blocks
+
+    // checkpoint step 3 over the scores of all ranks: every rank runs the same deterministic selection.  Lengths
+    // play no part here, so the global layout is taken as blocks of one element.
+    Geom gg{};
+    gg.n_elems = n_global_blocks;
+    gg.row_len = 1;
+    gg.n_blocks = n_global_blocks;
+    gg.block_elems = 1;
+    gg.blocks_per_row = 1;
+    gg.n_shards = 1;
+    gg.vec_ok = 0;
+    rc = c->dt == SCAR_F32
+             ? launch_select<float>(c, static_cast<const float *>(d_global_scores), gg, k_global, c->glob, false)
+             : launch_select<unsigned long long>(c, static_cast<const unsigned long long *>(d_global_scores), gg,
+                                                 k_global, c->glob, false);
+    if (rc != SCAR_OK) {
+        cudaGetLastError();
+        return rc;
+    }
+    // which of the chosen blocks are this rank's, and how many
+    CU_TRY(cudaMemsetAsync(c->member, 0, B * 4, c->stream));
+    CU_TRY(cudaMemsetAsync(c->d_count, 0, 3 * 8, c->stream));
+    if (k_global) {
+        k_mark_members<<<(unsigned)((k_global + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(
+            c->glob.sel, c->glob.info, first_block, B, c->member, c->d_count);
+        ++c->launches;
+    }
+    CU_TRY(cudaMemcpyAsync(c->h_count, c->d_count, 3 * 8, cudaMemcpyDeviceToHost, c->stream));
+    CU_TRY(cudaStreamSynchronize(c->stream));
+    if (c->h_count[1]) {
+        CU_TRY(cudaMemsetAsync(&c->glob.info->error, 0, sizeof(unsigned long long), c->stream));
+        return SCAR_ERR_TIMEOUT;
+    }
+    const uint64_t k_local = c->h_count[0], nonfinite = c->h_count[2];
+    // checkpoint step 4 on this rank's own blocks: the marks serve as priorities, so the k_local marked blocks are
+    // exactly the k_local largest, and the usual selection + pack writes ids, offsets, payload and refreshes z
+    rc = enqueue_baseline_save(c, k_local, c->member);
+    if (rc != SCAR_OK) return rc;
+    rc = fetch_save(c, out);
+    if (rc == SCAR_OK) out->nonfinite_blocks = nonfinite;
+    return rc;
 }
 
 int scar_ckpt_save_round(scar_ctx *c, uint64_t k, scar_save_info *out) {

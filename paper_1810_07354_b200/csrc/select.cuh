@@ -892,6 +892,32 @@ k_full_save(const T *__restrict__ x, T *__restrict__ z, T *__restrict__ payload,
     }
 }
 
+// ---- multi-GPU form of a save: which of the globally selected blocks are this rank's ---------------
+//
+// sel_g holds the ascending global ids chosen among all ranks' scores.  Marks, in member[0..n_local), the ones in
+// [first, first + n_local) (member must be zero before) and counts them; rec = {count, error of the global
+// selection, non-finite scores over all ranks} for the host.
+static __global__ void __launch_bounds__(kThreads)
+k_mark_members(const uint32_t *__restrict__ sel_g, const SaveInfoDev *info_g, unsigned long long first,
+               unsigned long long n_local, uint32_t *__restrict__ member, unsigned long long *rec) {
+    const unsigned long long j = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
+    const bool failed = info_g->error != 0;
+    bool mine = false;
+    if (!failed && j < info_g->k) {
+        const unsigned long long id = sel_g[j];
+        if (id >= first && id - first < n_local) {
+            member[id - first] = 1u;
+            mine = true;
+        }
+    }
+    const unsigned bal = __ballot_sync(0xffffffffu, mine);
+    if ((threadIdx.x & 31) == 0 && bal) atomicAdd(&rec[0], (unsigned long long)__popc(bal));
+    if (j == 0) {
+        rec[1] = info_g->error;
+        rec[2] = info_g->nonfinite_blocks;
+    }
+}
+
 // ---- baseline strategies of Section 5.4 -------------------------------------
 //
 // `round`: the k blocks that follow a cursor, wrapping at the end of the buffer.

@@ -92,8 +92,9 @@ class Simulation:
         assert self.strategy in STRATEGIES and 0.0 < self.r <= 1.0
         self.ck = api.ScarCheckpoint(self.x, n_shards=1, block_elems=self.block)  # z := x^(0), Section 4.2
         self.n_blocks = self.ck.n_blocks
-        self.k = max(1, min(self.n_blocks, int(math.floor(self.r * self.n_blocks + 0.5))))
-        self.period = max(1, int(math.floor(self.r * self.full_period + 0.5)))
+        # blocks per save and iterations between saves: both by the library's own rounding rule for a fraction
+        self.k = api.scar_k_from_r(self.r, self.n_blocks)
+        self.period = api.scar_k_from_r(self.r, self.full_period)
         self._gen = torch.Generator(device=self.x.device).manual_seed(self.seed)
 
     def draw_priorities(self):

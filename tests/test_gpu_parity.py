@@ -518,6 +518,37 @@ def test_a_barrier_that_cannot_complete_times_out_and_the_context_survives(kind)
     ck.close()
 
 
+def test_many_shard_runs_can_be_captured_and_replayed_with_the_mask_of_the_capture():
+    """64 alternating lost shards do not fit the launch parameters as runs, so the shard flags travel by value
+    inside the expansion kernel's parameters: nothing reads the caller's array after the call returns, and a
+    captured recovery replays with the mask it was captured with even after that array has changed."""
+    w = make_workload("tiny", n_elems=1 << 18, block_elems=64)  # 4096 blocks
+    boff = block_offsets(w.geom)
+    s = torch.cuda.Stream()
+    x = parity.to_dev(w.x)
+    x0 = x.clone()
+    torch.cuda.synchronize()
+    ck = api.ScarCheckpoint(x, n_shards=64, block_elems=64, stream=s)
+    ck.load(parity.to_dev(w.z))
+    torch.cuda.synchronize()
+    m = np.zeros(64, dtype=np.uint8)
+    m[::2] = 1
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        ck.recover_partial(m, sync=False)
+    want, x_after = oracle.recover_partial(w.x, w.z, boff, oracle.expand_shards(w.n_blocks, m))
+    m[:] = 0  # the caller's array is its own again
+    for _ in range(2):
+        x.copy_(x0)
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        _, nrm = api.scar_ckpt_last_info(ck.ctx, False, True)
+        parity.check_norm(nrm, want, True)
+        assert x.cpu().numpy().tobytes() == x_after.tobytes()
+    ck.close()
+
+
 # ------------------------------------------------------------------ several contexts at once
 
 

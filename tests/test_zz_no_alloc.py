@@ -14,7 +14,8 @@ import ctypes as C
 import numpy as np
 import pytest
 
-from workloads import make_workload
+import oracle
+from workloads import Geometry, block_offsets, make_workload
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -63,7 +64,13 @@ def test_static_norm_matches_context_norm_on_two_calls_in_a_row(name, kw):
         api.scar_perturbation_norm_static(x, z, dt, layout, m, d_out, stream)
         torch.cuda.synchronize()
         got.append(read_info(d_out))
-    assert torch.cuda.mem_get_info()[0] == free_before, "the call must not change device memory in use"
+    # the figure is device-wide (other processes may free memory meanwhile): it must not have gone down
+    assert torch.cuda.mem_get_info()[0] >= free_before, "the call must not take device memory"
+    boff = block_offsets(w.geom)
+    for g, m in zip(got, masks):  # and against the definition itself, not only against the other entry point
+        ora = oracle.perturbation_norm(w.x, w.z, boff, None if m is None else m.cpu().numpy())
+        assert (g.lost_blocks, g.lost_elems, g.l1) == (ora.lost_blocks, ora.lost_elems, ora.l1)
+        assert abs(g.l2 - ora.l2) <= 1e-5 * ora.l2
     for g, wnt in zip(got, want):
         assert (g.lost_blocks, g.lost_elems, g.l1) == (wnt.lost_blocks, wnt.lost_elems, wnt.l1)
         if is_float:
@@ -73,6 +80,55 @@ def test_static_norm_matches_context_norm_on_two_calls_in_a_row(name, kw):
             assert g.l2 == 0.0
     # inputs are read-only
     assert x.cpu().numpy().tobytes() == w.x.tobytes() and z.cpu().numpy().tobytes() == w.z.tobytes()
+
+
+@pytest.mark.parametrize("n,row,blk", [
+    (1001 * 37, 1001, 256),     # rows of 1001 floats: element-wise path, last block of a row shorter
+    (100_000 * 12, 100_000, 1024),  # MLR-shaped rows: 97 full blocks and a tail of 672
+    (1 << 20, 0, 1),            # exactly the largest block count the static array holds
+])
+def test_static_norm_on_other_geometries_twice_in_a_row(n, row, blk):
+    """The entry point resolves the geometry and picks its launch shape itself: rows whose last block is
+    shorter, blocks that are not 16-byte aligned, and a layout of exactly SCAR_STATIC_MAX_BLOCKS blocks, each
+    called twice through the shared array and compared with the context-based call and with the definition."""
+    r = np.random.Generator(np.random.PCG64(n + blk))
+    geom = Geometry(n, row, blk, 1)
+    zh = r.standard_normal(n).astype(np.float32)
+    xh = (zh + r.standard_normal(n).astype(np.float32) * np.float32(0.05)).astype(np.float32)
+    boff = block_offsets(geom)
+    nb = boff.size - 1
+    x, z = torch.from_numpy(xh).cuda(), torch.from_numpy(zh).cuda()
+    layout = api.make_layout(n, row, blk, 1)
+    d_out = torch.zeros(4, dtype=torch.int64, device="cuda")
+    for mask_h in ((r.random(nb) < 0.5).astype(np.uint8), None):
+        m = None if mask_h is None else torch.from_numpy(mask_h).cuda()
+        want = reference(x, z, geom, m, True)
+        ora = oracle.perturbation_norm(xh, zh, boff, mask_h)
+        for _ in range(2):
+            api.scar_perturbation_norm_static(x, z, api.SCAR_F32, layout, m, d_out)
+            torch.cuda.synchronize()
+            g = read_info(d_out)
+            assert (g.lost_blocks, g.lost_elems) == (want.lost_blocks, want.lost_elems) == (ora.lost_blocks, ora.lost_elems)
+            assert g.l2 == want.l2 and abs(g.l2 - ora.l2) <= 1e-5 * ora.l2
+
+
+def test_a_warmed_up_static_call_changes_nothing_it_should_not():
+    """A zero-size call is a complete warm-up (it looks the array's address up and loads the module that holds
+    it); after it, a real call leaves device memory in use as it was."""
+    d_out = torch.ones(4, dtype=torch.int64, device="cuda")
+    empty = api.make_layout(0, 0, 256, 1)
+    api.scar_perturbation_norm_static(None, None, api.SCAR_F32, empty, None, d_out)
+    torch.cuda.synchronize()
+    assert d_out.cpu().tolist() == [0, 0, 0, 0]
+    buf = torch.arange(1 << 14, dtype=torch.float32, device="cuda")
+    zero = torch.zeros(1 << 14, dtype=torch.float32, device="cuda")
+    before = torch.cuda.mem_get_info()[0]
+    api.scar_perturbation_norm_static(buf, zero, api.SCAR_F32, api.make_layout(1 << 14, 0, 128, 1), None, d_out)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] >= before
+    info = read_info(d_out)
+    want = float(np.sqrt(np.sum(np.arange(1 << 14, dtype=np.float64) ** 2)))
+    assert abs(info.l2 - want) <= 1e-5 * want and info.lost_blocks == 128
 
 
 def test_static_norm_rejects_what_it_cannot_hold():
