@@ -391,6 +391,23 @@ double scar_irreducible_error(double delta_max, double c);
  * SCAR_ERR_STATE on an empty buffer. */
 int scar_ckpt_selftest_arm_timeout(scar_ctx *ctx);
 
+/* ---- Guard bands (debugging aid; no counterpart in the paper) ------------------
+ * scar_ckpt_init_guarded is scar_ckpt_init for a context whose every device
+ * buffer (running checkpoint, payload, scores, id and offset lists, masks,
+ * selection and reduction scratch, segment tables, drain and sharding buffers
+ * allocated later) sits between two bands of 256 bytes holding a known pattern,
+ * the second band starting at the first byte behind the buffer.
+ * scar_ckpt_debug_check_guards waits for the stream and counts, on the device,
+ * the band bytes that no longer hold the pattern: any write of the library's
+ * kernels just outside one of its buffers shows up as a non-zero count.
+ * SCAR_ERR_STATE on a context that was not created guarded.
+ * scar_static_debug_check_guard does the same for the band behind the fixed
+ * array of scar_perturbation_norm_static on the current device (waits for the
+ * device; SCAR_ERR_STATE before that call was ever used there). */
+int scar_ckpt_init_guarded(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *layout, void *cuda_stream);
+int scar_ckpt_debug_check_guards(scar_ctx *ctx, uint64_t *bad_bytes);
+int scar_static_debug_check_guard(uint64_t *bad_bytes);
+
 /* Diagnostic builds only (library compiled with -DSCAR_SELECT_STAMPS; otherwise
  * SCAR_ERR_STATE).  Waits for the stream and copies the 32 time stamps of the
  * most recent selection kernel: SM clock cycles of its first CTA at

@@ -62,6 +62,9 @@ def exported_symbols() -> list:
 _vp, _u64, _int, _dbl = C.c_void_p, C.c_uint64, C.c_int, C.c_double
 _SIGS = {
     "scar_ckpt_init": (_int, [C.POINTER(_vp), _vp, _int, C.POINTER(scar_layout), _vp]),
+    "scar_ckpt_init_guarded": (_int, [C.POINTER(_vp), _vp, _int, C.POINTER(scar_layout), _vp]),
+    "scar_ckpt_debug_check_guards": (_int, [_vp, C.POINTER(_u64)]),
+    "scar_static_debug_check_guard": (_int, [C.POINTER(_u64)]),
     "scar_ckpt_set_norm": (_int, [_vp, _int, _vp]),
     "scar_ckpt_block_scores": (_int, [_vp]),
     "scar_ckpt_priority_save": (_int, [_vp, _dbl, C.POINTER(scar_save_info)]),
@@ -157,11 +160,29 @@ def make_layout(n_elems: int, row_elems: int = 0, block_elems: int = 0, n_shards
     return L
 
 
-def scar_ckpt_init(d_x, dtype: int, layout: scar_layout, cuda_stream: int = 0) -> int:
+def scar_ckpt_init(d_x, dtype: int, layout: scar_layout, cuda_stream: int = 0, guarded: bool = False) -> int:
     ctx = _vp()
-    _check(load_library().scar_ckpt_init(C.byref(ctx), _addr(d_x), dtype, C.byref(layout), cuda_stream or None),
-           "scar_ckpt_init")
+    name = "scar_ckpt_init_guarded" if guarded else "scar_ckpt_init"
+    _check(getattr(load_library(), name)(C.byref(ctx), _addr(d_x), dtype, C.byref(layout), cuda_stream or None), name)
     return ctx.value
+
+
+def scar_ckpt_init_guarded(d_x, dtype: int, layout: scar_layout, cuda_stream: int = 0) -> int:
+    """``scar_ckpt_init`` for a debug context whose device buffers sit between guard bands."""
+    return scar_ckpt_init(d_x, dtype, layout, cuda_stream, guarded=True)
+
+
+def scar_ckpt_debug_check_guards(ctx: int) -> int:
+    """Band bytes of a guarded context that no longer hold the pattern (0 = nothing wrote outside a buffer)."""
+    bad = _u64(0)
+    _check(load_library().scar_ckpt_debug_check_guards(ctx, C.byref(bad)), "scar_ckpt_debug_check_guards")
+    return int(bad.value)
+
+
+def scar_static_debug_check_guard() -> int:
+    bad = _u64(0)
+    _check(load_library().scar_static_debug_check_guard(C.byref(bad)), "scar_static_debug_check_guard")
+    return int(bad.value)
 
 
 def scar_ckpt_set_norm(ctx: int, norm: int, h_block_weights: Optional[np.ndarray] = None) -> None:
@@ -420,17 +441,18 @@ class ScarCheckpoint:
     """One context over a torch CUDA tensor ``x`` (float32 or int32, flat, contiguous)."""
 
     def __init__(self, x, n_shards: int = 8, row_elems: int = 0, block_elems: int = 0,
-                 block_offsets: Optional[np.ndarray] = None, stream=None):
+                 block_offsets: Optional[np.ndarray] = None, stream=None, guarded: bool = False):
         import torch
 
         assert x.is_cuda and x.is_contiguous() and x.dim() == 1
         self.dtype = {torch.float32: SCAR_F32, torch.int32: SCAR_I32}[x.dtype]
+        self.guarded = guarded
         self.x = x
         self.n_elems = x.numel()
         self._stream = stream if stream is not None else torch.cuda.current_stream(x.device)
         self._layout = make_layout(self.n_elems, row_elems, block_elems, n_shards, block_offsets)
         with torch.cuda.device(x.device):
-            self.ctx = scar_ckpt_init(x, self.dtype, self._layout, self._stream.cuda_stream)
+            self.ctx = scar_ckpt_init(x, self.dtype, self._layout, self._stream.cuda_stream, guarded)
         self.n_blocks = scar_ckpt_n_blocks(self.ctx)
 
     # views -----------------------------------------------------------------
@@ -452,6 +474,9 @@ class ScarCheckpoint:
         if block_weights is not None:
             assert len(block_weights) == self.n_blocks
         scar_ckpt_set_norm(self.ctx, norm, block_weights)
+
+    def check_guards(self) -> int:
+        return scar_ckpt_debug_check_guards(self.ctx)
 
     def block_scores(self):
         scar_ckpt_block_scores(self.ctx)

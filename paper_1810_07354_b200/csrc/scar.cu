@@ -107,6 +107,16 @@ struct scar_ctx {
     std::vector<uint64_t> longest_prefix;  // explicit layouts: [k] = elements of the k longest blocks
     char *io_stage = nullptr;      // pinned staging buffer for whole-checkpoint transfers
 
+    // debug contexts (scar_ckpt_init_guarded): every device allocation sits between two bands of kGuardBytes
+    // bytes of a known pattern
+    bool guarded = false;
+    struct Band {
+        const uint8_t *user;  // the buffer the library uses
+        size_t bytes;         // its size: the bands are [user - kGuardBytes, user) and [user + bytes, + kGuardBytes)
+    };
+    std::vector<Band> bands;
+    unsigned long long *d_bad = nullptr;  // result of the guard check
+
     std::vector<void *> owned;  // device allocations to free
     std::vector<void *> owned_host;  // pinned host allocations to free
     uint64_t launches = 0;
@@ -132,15 +142,53 @@ int check_device(const scar_ctx *c) {
     return dev == c->device ? SCAR_OK : SCAR_ERR_STATE;
 }
 
+constexpr size_t kGuardBytes = 256;  // keeps guarded buffers 256-byte aligned, like cudaMalloc's own
+constexpr int kGuardPattern = 0xA5;
+
 template <typename P> int dev_alloc(scar_ctx *c, P **p, size_t bytes) {
     void *q = nullptr;
-    if (cudaMalloc(&q, bytes ? bytes : 16) != cudaSuccess) {
+    if (bytes == 0) bytes = 16;
+    if (!c->guarded) {
+        if (cudaMalloc(&q, bytes) != cudaSuccess) {
+            cudaGetLastError();
+            return SCAR_ERR_ALLOC;
+        }
+        c->owned.push_back(q);
+        *p = static_cast<P *>(q);
+        return SCAR_OK;
+    }
+    // the tail band starts at the first byte behind the buffer, so an overrun of a single element lands in it
+    if (cudaMalloc(&q, bytes + 2 * kGuardBytes) != cudaSuccess) {
         cudaGetLastError();
         return SCAR_ERR_ALLOC;
     }
     c->owned.push_back(q);
-    *p = static_cast<P *>(q);
+    uint8_t *user = static_cast<uint8_t *>(q) + kGuardBytes;
+    if (cudaMemsetAsync(q, kGuardPattern, kGuardBytes, c->stream) != cudaSuccess ||
+        cudaMemsetAsync(user + bytes, kGuardPattern, kGuardBytes, c->stream) != cudaSuccess)
+        return SCAR_ERR_CUDA;
+    c->bands.push_back({user, bytes});
+    *p = reinterpret_cast<P *>(user);
     return SCAR_OK;
+}
+
+// One CTA per buffer: counts the bytes of its two bands that no longer hold the pattern.
+constexpr int kBandsPerLaunch = 48;
+struct BandList {
+    const uint8_t *user[kBandsPerLaunch];
+    unsigned long long bytes[kBandsPerLaunch];
+};
+__global__ void __launch_bounds__(kThreads)
+k_check_guards(BandList list, unsigned long long *bad) {
+    const uint8_t *user = list.user[blockIdx.x];
+    unsigned wrong = 0;
+    for (unsigned i = threadIdx.x; i < 2 * kGuardBytes; i += kThreads) {
+        const uint8_t v = i < kGuardBytes ? user[(long long)i - (long long)kGuardBytes]
+                                          : user[list.bytes[blockIdx.x] + (i - kGuardBytes)];
+        wrong += v != (uint8_t)kGuardPattern;
+    }
+    wrong = __reduce_add_sync(0xffffffffu, wrong);
+    if ((threadIdx.x & 31) == 0 && wrong) atomicAdd(bad, (unsigned long long)wrong);
 }
 
 // Validates the caller's layout and fills the host-side fields of Geom
@@ -768,7 +816,8 @@ void destroy_impl(scar_ctx *c) {
 
 extern "C" {
 
-int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *layout, void *cuda_stream) {
+static int init_impl(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *layout, void *cuda_stream,
+                     bool guarded) {
     if (!out) return SCAR_ERR_INVALID_ARG;
     *out = nullptr;
     if (!layout || (dt != SCAR_F32 && dt != SCAR_I32)) return SCAR_ERR_INVALID_ARG;
@@ -787,6 +836,7 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     if (!c) return SCAR_ERR_ALLOC;
     c->device = dev;
     c->stream = static_cast<cudaStream_t>(cuda_stream);
+    c->guarded = guarded;
     c->dt = dt;
     c->g = g;
     c->x = d_x;
@@ -913,6 +963,46 @@ int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *
     }
     c->last = c->cur;
     *out = c;
+    return SCAR_OK;
+}
+
+int scar_ckpt_init(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *layout, void *cuda_stream) {
+    return init_impl(out, d_x, dt, layout, cuda_stream, false);
+}
+
+int scar_ckpt_init_guarded(scar_ctx **out, void *d_x, scar_dtype dt, const scar_layout *layout, void *cuda_stream) {
+    return init_impl(out, d_x, dt, layout, cuda_stream, true);
+}
+
+int scar_ckpt_debug_check_guards(scar_ctx *c, uint64_t *bad_bytes) {
+    if (!c || !bad_bytes) return SCAR_ERR_INVALID_ARG;
+    if (!c->guarded) return SCAR_ERR_STATE;
+    int rc = check_device(c);
+    if (rc != SCAR_OK) return rc;
+    if (!c->d_bad) {
+        void *q = nullptr;  // not through dev_alloc: the list of bands must not change while it is walked
+        if (cudaMalloc(&q, 8) != cudaSuccess) {
+            cudaGetLastError();
+            return SCAR_ERR_ALLOC;
+        }
+        c->owned.push_back(q);
+        c->d_bad = static_cast<unsigned long long *>(q);
+    }
+    CU_TRY(cudaMemsetAsync(c->d_bad, 0, 8, c->stream));
+    for (size_t i = 0; i < c->bands.size(); i += kBandsPerLaunch) {
+        BandList list{};
+        const size_t n = c->bands.size() - i < (size_t)kBandsPerLaunch ? c->bands.size() - i : (size_t)kBandsPerLaunch;
+        for (size_t j = 0; j < n; ++j) {
+            list.user[j] = c->bands[i + j].user;
+            list.bytes[j] = c->bands[i + j].bytes;
+        }
+        k_check_guards<<<(unsigned)n, kThreads, 0, c->stream>>>(list, c->d_bad);
+    }
+    CU_TRY(cudaGetLastError());
+    unsigned long long bad = 0;
+    CU_TRY(cudaMemcpyAsync(&bad, c->d_bad, 8, cudaMemcpyDeviceToHost, c->stream));
+    CU_TRY(cudaStreamSynchronize(c->stream));
+    *bad_bytes = bad;
     return SCAR_OK;
 }
 

@@ -30,10 +30,14 @@ constexpr uint64_t kStaticMaxBlocks = SCAR_STATIC_MAX_BLOCKS;
 constexpr uint64_t kStaticMaxCtas = kStaticMaxBlocks / (kThreads / 4) + 1;
 // 8-byte words: three slots per CTA, three per watcher.
 constexpr uint64_t kScratchWords = 3 * kStaticMaxCtas + 3 * kMaxWatchers;
+// Behind them, a band of words that nothing may write: it is filled with a pattern when the address is looked up
+// and scar_static_debug_check_guard counts the bytes that have changed since.
+constexpr uint64_t kGuardWords = 32;
+constexpr int kGuardPattern = 0xA5;
 
 // In host code this name is only a handle for cudaGetSymbolAddress: it is not
 // a device address and must never be passed to a kernel as one.
-static __device__ __align__(256) unsigned long long g_static_scratch[kScratchWords];
+static __device__ __align__(256) unsigned long long g_static_scratch[kScratchWords + kGuardWords];
 
 constexpr int kMaxDevices = 64;
 std::mutex g_mu;
@@ -41,7 +45,7 @@ unsigned long long *g_scratch_addr[kMaxDevices] = {};
 
 // Device address of the scratch array on the current device, looked up once
 // per device (with that device current) and remembered.
-int scratch_on_current_device(unsigned long long **out) {
+int scratch_on_current_device(unsigned long long **out, cudaStream_t stream) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return SCAR_ERR_CUDA;
     if (dev < 0 || dev >= kMaxDevices) return SCAR_ERR_STATE;
@@ -52,6 +56,9 @@ int scratch_on_current_device(unsigned long long **out) {
             cudaGetLastError();
             return SCAR_ERR_CUDA;
         }
+        if (cudaMemsetAsync(static_cast<unsigned long long *>(p) + kScratchWords, kGuardPattern, kGuardWords * 8, stream) !=
+            cudaSuccess)
+            return SCAR_ERR_CUDA;
         g_scratch_addr[dev] = static_cast<unsigned long long *>(p);
     }
     *out = g_scratch_addr[dev];
@@ -105,7 +112,7 @@ extern "C" int scar_perturbation_norm_static(const void *d_x, const void *d_z, s
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     // Looked up first, so that even a call on an empty layout is a complete warm-up of this device.
     unsigned long long *scratch = nullptr;
-    int rc = scratch_on_current_device(&scratch);
+    int rc = scratch_on_current_device(&scratch, stream);
     if (rc != SCAR_OK) return rc;
     if (layout->n_elems == 0)
         return cudaMemsetAsync(d_out, 0, sizeof(scar_norm_info), stream) == cudaSuccess ? SCAR_OK : SCAR_ERR_CUDA;
@@ -133,4 +140,24 @@ extern "C" int scar_perturbation_norm_static(const void *d_x, const void *d_z, s
 
     return dt == SCAR_F32 ? run_static<float>(d_x, d_z, g, S, scratch, d_out, stream)
                           : run_static<int>(d_x, d_z, g, S, scratch, d_out, stream);
+}
+
+extern "C" int scar_static_debug_check_guard(uint64_t *bad_bytes) {
+    if (!bad_bytes) return SCAR_ERR_INVALID_ARG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SCAR_ERR_CUDA;
+    unsigned long long *base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (dev < 0 || dev >= kMaxDevices || !g_scratch_addr[dev]) return SCAR_ERR_STATE;  // never used on this device
+        base = g_scratch_addr[dev];
+    }
+    unsigned char tail[kGuardWords * 8];
+    if (cudaDeviceSynchronize() != cudaSuccess ||
+        cudaMemcpy(tail, base + kScratchWords, sizeof tail, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return SCAR_ERR_CUDA;
+    uint64_t bad = 0;
+    for (unsigned char b : tail) bad += b != (unsigned char)kGuardPattern;
+    *bad_bytes = bad;
+    return SCAR_OK;
 }

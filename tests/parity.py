@@ -30,11 +30,14 @@ def to_dev(a: np.ndarray) -> torch.Tensor:
 
 
 def make_ctx(x_dev: torch.Tensor, z_host: np.ndarray, geom=None, boff=None, n_shards=8) -> api.ScarCheckpoint:
-    """Context over ``x_dev`` whose running checkpoint is then replaced by ``z_host``."""
+    """Context over ``x_dev`` whose running checkpoint is then replaced by ``z_host``.  The context is a guarded
+    one: every buffer the library allocates sits between two bands of a known pattern, and ``close`` (see
+    conftest.py) fails the test when a kernel has written into a band."""
     if boff is not None:
-        ck = api.ScarCheckpoint(x_dev, n_shards=n_shards, block_offsets=boff)
+        ck = api.ScarCheckpoint(x_dev, n_shards=n_shards, block_offsets=boff, guarded=True)
     else:
-        ck = api.ScarCheckpoint(x_dev, n_shards=geom.n_shards, row_elems=geom.row_elems, block_elems=geom.block_elems)
+        ck = api.ScarCheckpoint(x_dev, n_shards=geom.n_shards, row_elems=geom.row_elems, block_elems=geom.block_elems,
+                                guarded=True)
     if z_host is not None:
         zt = to_dev(z_host)
         ck.load(zt)

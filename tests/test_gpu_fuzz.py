@@ -83,7 +83,7 @@ def test_random_case(seed):
     nb = boff.size - 1
     is_float = x.dtype == np.float32
     xd = parity.to_dev(x)
-    ck = api.ScarCheckpoint(xd, **layout)
+    ck = api.ScarCheckpoint(xd, guarded=True, **layout)  # every library buffer between two guard bands
     assert ck.n_blocks == nb
     ck.load(parity.to_dev(z))
     if norm == "l1" or w is not None:
@@ -129,4 +129,5 @@ def test_random_case(seed):
     _, x_after = oracle.recover_partial(x, hz, boff, lost)
     assert xd.cpu().numpy().tobytes() == x_after.tobytes()
     assert parity.same_bits(ck.views()["z"].cpu().numpy(), hz)
+    assert ck.check_guards() == 0, "a kernel wrote just outside one of the library's buffers"
     ck.close()

@@ -627,3 +627,35 @@ def test_enqueue_only_calls_can_be_captured_in_a_cuda_graph():
         parity.check_norm(nrm, want, True)
         assert x.cpu().numpy().tobytes() == x_after.tobytes()
     ck.close()
+
+
+# ------------------------------------------------------------------ guard bands
+
+
+def test_guard_bands_notice_a_single_element_written_outside_a_buffer():
+    """The checker itself: a guarded context reports clean bands after a save and a recovery, and reports the
+    damage when one element right behind the running checkpoint (inside the allocation's own guard band, so the
+    write is harmless) is overwritten."""
+    w = make_workload("mf", l_rows=3000, r_rows=100)
+    xd = parity.to_dev(w.x)
+    ck = api.ScarCheckpoint(xd, n_shards=4, row_elems=w.geom.row_elems, block_elems=w.geom.block_elems, guarded=True)
+    ck.load(parity.to_dev(w.z))
+    ck.priority_save(0.3)
+    ck.recover_partial_blocks(parity.to_dev(w.lost_blocks))
+    assert ck.check_guards() == 0
+    n = w.x.size
+    z_addr = api.scar_ckpt_view(ck.ctx)["z"]
+    behind = api.device_array(z_addr + 4 * n, 1, np.float32)  # first element of the band behind z
+    before = behind.clone()
+    behind.fill_(1.0)
+    torch.cuda.synchronize()
+    assert ck.check_guards() == 4
+    behind.copy_(before)
+    torch.cuda.synchronize()
+    assert ck.check_guards() == 0
+    plain = api.ScarCheckpoint(parity.to_dev(w.x), block_elems=w.geom.block_elems)
+    with pytest.raises(api.ScarError) as e:
+        plain.check_guards()
+    assert e.value.code == -5
+    plain.close()
+    ck.close()

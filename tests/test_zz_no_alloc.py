@@ -151,3 +151,8 @@ def test_static_norm_rejects_what_it_cannot_hold():
     torch.cuda.synchronize()
     info = read_info(d_out)
     assert info.l2 == 0.0 and info.lost_blocks == 16 and info.lost_elems == 1 << 12
+
+
+def test_nothing_was_written_behind_the_static_array():
+    """Runs after the calls above: the band behind the library's fixed array still holds its pattern."""
+    assert api.scar_static_debug_check_guard() == 0
