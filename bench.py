@@ -311,6 +311,25 @@ def device_workload(name, n_elems, rank, dev):
             w.lost_blocks)
 
 
+class L2Flush:
+    """Empties the L2 cache of everything a timed call could reuse: writes a 256 MiB buffer (twice the 126 MB
+    L2), then reads another 256 MiB one.  The read pass matters for the small parameter sets: a write-only flush
+    leaves the cache full of the flush buffer's dirty lines, and the next call then pays for writing them back
+    (up to 126 MB of foreign DRAM traffic inside a call that itself moves 150 to 900 MB); after the read pass the
+    cache holds clean lines that are dropped for free.  Always outside the timed intervals."""
+
+    def __init__(self, dev):
+        import torch
+
+        self.w = torch.empty(64 << 20, dtype=torch.float32, device=dev)
+        self.r = torch.zeros(64 << 20, dtype=torch.float32, device=dev)
+        self.sink = None
+
+    def zero_(self):
+        self.w.zero_()
+        self.sink = self.r.sum()
+
+
 class Measured:
     """Raw results of the timed steps of one workload on this rank."""
 
@@ -338,7 +357,7 @@ def measure_workload(api, name, n_elems, rank, dev, steps, warmup, barrier):
         return ck.recover_partial(lost_shards, sync=sync)
 
     m.z_lib = z_lib = ck.views()["z"]  # the library's running checkpoint, aliased (no copy)
-    m.flush = flush = torch.empty(64 << 20, dtype=torch.float32, device=dev)  # 256 MiB, larger than the 126 MB L2
+    m.flush = flush = L2Flush(dev)
 
     def reset_checkpoint():
         """Pristine running checkpoint, then an L2 flush; plain torch copies, outside every timed interval."""
@@ -492,7 +511,7 @@ def run_gpu(args):
     summ = summarise(m, peak)
     achieved = scanned / (m.score_ms * 1e-3) / 1e9
     l2_note = ("inputs larger than L2; " if scanned > (512 << 20) else "inputs NOT larger than L2; ") + \
-        "L2 flushed by a 256 MiB write after every untimed state reset and before every timed call"
+        "L2 flushed by a 256 MiB write followed by a 256 MiB read after every untimed state reset and before every timed call"
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -586,7 +605,7 @@ def run_sharded(args):
     x = x0.clone()
     sc = ShardedCheckpoint(x, nb_global, world, rank, n_shards=8, block_elems=BLOCK)
     z_lib = sc.ck.views()["z"]
-    flush = torch.empty(64 << 20, dtype=torch.float32, device=dev)
+    flush = L2Flush(dev)
     r_sweep = (0.01, 0.1, 0.5, 1.0)
     ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
 
@@ -662,6 +681,44 @@ def run_sharded(args):
     sc.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_select_stamps(args):
+    """Where the selection kernel's time goes: with a diagnostic build of the library
+    (``python -m paper_1810_07354_b200._build --select-stamps``) prints, per r of the workload, the microseconds
+    between the marked points of the kernel's first CTA (median of 8 saves; SM cycles / the SM clock in MHz).
+    Rebuild without the flag afterwards."""
+    import torch
+
+    from paper_1810_07354_b200 import api
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    geom, z0, x0, r_sweep, _, _ = device_workload(args.workload, args.n_elems, 0, dev)
+    ck = api.ScarCheckpoint(x0.clone(), n_shards=geom.n_shards, row_elems=geom.row_elems, block_elems=geom.block_elems)
+    mhz = float(subprocess.run(["nvidia-smi", "-i", "0", "--query-gpu=clocks.max.sm", "--format=csv,noheader,nounits"],
+                               capture_output=True, text=True).stdout.split()[0])
+    flush = L2Flush(dev)
+    out = {"workload": args.workload, "n_blocks": ck.n_blocks, "sm_mhz_assumed": mhz, "per_r": {}}
+    for r in r_sweep:
+        runs = []
+        for _ in range(10):
+            ck.load(z0)
+            flush.zero_()
+            ck.priority_save(r)
+            runs.append(api.scar_ckpt_debug_select_stamps(ck.ctx))
+        st = np.median(np.array(runs[2:], dtype=np.float64), axis=0)
+        us = lambda a, b: round(float(st[b] - st[a]) / mhz, 2)  # noqa: E731
+        rec, last = {"keys_loaded": us(0, 1)}, 1
+        for p in range(6):
+            if st[2 + 4 * p] > st[0]:  # this digit pass ran
+                rec[f"pass{p}"] = {"histogram": us(last, 2 + 4 * p), "flush": us(2 + 4 * p, 3 + 4 * p),
+                                   "wait": us(3 + 4 * p, 4 + 4 * p), "resolve": us(4 + 4 * p, 5 + 4 * p)}
+                last = 5 + 4 * p
+        rec.update(counts=us(last, 26), exchange=us(26, 27), scan=us(27, 28), emit=us(28, 29), total=us(0, 29))
+        out["per_r"][str(r)] = rec
+    ck.close()
+    print(json.dumps(out))
 
 
 def run_extras(api, ck, x, x0, z_lib, z0, geom, r_sweep, flush, dev, with_bylayer):
@@ -829,6 +886,8 @@ def main():
     ap.add_argument("--sharded", action="store_true",
                     help="multi-GPU form of the save: the blocks of one parameter vector split over the ranks, "
                          "global top-r through one all-gather of the scores (strong scaling) instead of replicas")
+    ap.add_argument("--select-stamps", action="store_true",
+                    help="diagnostic builds of the library only: print where the selection kernel spends its time")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true",
@@ -838,6 +897,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.select_stamps:
+        run_select_stamps(args)
     elif args.sharded:
         run_sharded(args)
     else:

@@ -224,7 +224,7 @@ int scar_perturbation_norm_blocks(scar_ctx *ctx, const uint8_t *d_lost_blocks, s
  * that cannot take the device-wide synchronisation an allocation implies, or a
  * plug-in whose host forbids it to grow its memory.  This call needs no
  * context and calls no cudaMalloc / cudaFree or other allocating routine.  Its
- * partial sums live in a fixed array of about 0.4 MiB inside the library's
+ * partial sums live in a fixed array of about 0.3 MiB inside the library's
  * device image (every GPU that loads the library holds it until the process
  * exits), which caps the problem at SCAR_STATIC_MAX_BLOCKS blocks; larger
  * layouts return SCAR_ERR_CAPACITY and nothing is enqueued.

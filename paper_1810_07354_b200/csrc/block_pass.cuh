@@ -280,27 +280,25 @@ template <typename W> __device__ __forceinline__ W cta_sum(W v, W *sh) {
     return t;
 }
 
-// Scratch of the reduction: one slot per CTA of the pass and one per watcher.  A slot holds kSlotEmpty except
+// Scratch of the reduction: two slots per CTA of the pass and three per watcher.  A slot holds kSlotEmpty except
 // between its owner's store and the watcher's read, so the value itself tells the reader that it has arrived
 // (an aligned 8-byte store is seen whole or not at all); no fence, ticket or atomic is involved.
 constexpr unsigned long long kSlotEmpty = ~0ull;
 constexpr unsigned kMaxWatchers = kThreads;
 struct NormScratch {
-    unsigned long long *cta_val;     // per CTA: sum of its blocks' partials (bits of a double, or a uint64)
-    unsigned long long *cta_blocks;  // per CTA: lost blocks it covered
-    unsigned long long *cta_elems;   // per CTA: their elements
-    unsigned long long *tile_val;    // the same per watcher, kMaxWatchers of each
-    unsigned long long *tile_blocks;
-    unsigned long long *tile_elems;
+    unsigned long long *cta_val;   // per CTA: sum of its blocks' partials (bits of a double, or a uint64)
+    unsigned long long *cta_cnt;   // per CTA: lost blocks it covered (top 16 bits) and their elements (low 48)
+    unsigned long long *tile_val;  // per watcher, kMaxWatchers of each: the sum over its CTAs,
+    unsigned long long *tile_blocks;  // their lost blocks,
+    unsigned long long *tile_elems;   // and elements
 };
-// 8-byte words a launch of n_ctas CTAs needs: three arrays of n_ctas, then three of kMaxWatchers.
-inline size_t norm_scratch_words(uint64_t n_ctas) { return 3 * (size_t)n_ctas + 3 * kMaxWatchers; }
+// 8-byte words a launch of n_ctas CTAs needs: two arrays of n_ctas, then three of kMaxWatchers.
+inline size_t norm_scratch_words(uint64_t n_ctas) { return 2 * (size_t)n_ctas + 3 * kMaxWatchers; }
 inline NormScratch norm_scratch_at(unsigned long long *base, uint64_t n_ctas) {
     NormScratch rs;
     rs.cta_val = base;
-    rs.cta_blocks = base + n_ctas;
-    rs.cta_elems = base + 2 * n_ctas;
-    rs.tile_val = base + 3 * n_ctas;
+    rs.cta_cnt = base + n_ctas;
+    rs.tile_val = base + 2 * n_ctas;
     rs.tile_blocks = rs.tile_val + kMaxWatchers;
     rs.tile_elems = rs.tile_val + 2 * kMaxWatchers;
     return rs;
@@ -346,12 +344,38 @@ __device__ __forceinline__ void norm_write(NormInfoDev *out, bool is_float, bool
     out->lost_elems = ne;
 }
 
+// Sums a value (double for float data, else uint64) and a uint64 per thread over the CTA with one pair of
+// barriers, in a fixed order: xor tree inside each warp, then the warps in order.
+template <bool kF>
+__device__ __forceinline__ void cta_sum_pair(double &fs, unsigned long long &is, unsigned long long &cnt, double *shd,
+                                             unsigned long long *shu, unsigned long long *shc) {
+    if (kF) fs = group_sum<32, double>(fs);
+    else is = group_sum<32, unsigned long long>(is);
+    cnt = group_sum<32, unsigned long long>(cnt);
+    const int w = threadIdx.x >> 5;
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) {
+        if (kF) shd[w] = fs;
+        else shu[w] = is;
+        shc[w] = cnt;
+    }
+    __syncthreads();
+    fs = 0.0, is = 0, cnt = 0;
+#pragma unroll
+    for (int i = 0; i < kThreads / 32; ++i) {
+        if (kF) fs += shd[i];
+        else is += shu[i];
+        cnt += shc[i];
+    }
+}
+
 // Called by every thread of every CTA of a recovery / norm pass with the thread's own share (fs for float data,
-// is for integer data, lost blocks, lost elements).  The CTA's total goes to its slot with three plain stores,
-// and the CTA is done: nothing in the streaming part of the pass waits for the memory system on behalf of
-// the reduction.  The last CTAs of the grid (the watchers: one per 1024 CTAs) do the adding: watcher t collects
-// the slots of its contiguous share of the CTAs, thread i taking slots i, i + 256, ... in that order, then the
-// fixed tree of cta_sum; the last CTA collects the watchers' totals the same way and writes the result.
+// is for integer data, lost blocks, lost elements; a CTA covers fewer than 2^16 blocks and a buffer has fewer
+// than 2^48 elements, so the two counts travel in one word).  The CTA's total goes to its two slots with plain
+// stores, and the CTA is done: nothing in the streaming part of the pass waits for the memory system on behalf
+// of the reduction.  The last CTAs of the grid (the watchers: one per 1024 CTAs) do the adding: watcher t
+// collects the slots of its contiguous share of the CTAs, thread i taking slots i, i + 256, ... in that order,
+// then the fixed tree of cta_sum; the last CTA collects the watchers' totals the same way and writes the result.
 // A watcher only ever waits for CTAs with a lower index than its own, which were dispatched before it and wait
 // for nobody, and every wait is bounded.  The order of every addition depends only on the grid size, so the
 // result is the same bits on every run.  This replaces a second launch: the pass and its reduction are one kernel.
@@ -361,23 +385,22 @@ __device__ __forceinline__ void norm_epilogue(double fs, unsigned long long is, 
                                               bool take_sqrt) {
     typedef unsigned long long u64;
     constexpr bool kF = std::is_same<T, float>::value;
+    constexpr u64 kElemMask = (1ull << 48) - 1;
     __shared__ double shd[kThreads / 32];
     __shared__ u64 shu[kThreads / 32];
-    if (kF) fs = cta_sum<double>(fs, shd);
-    else is = cta_sum<u64>(is, shu);
-    nb = cta_sum<u64>(nb, shu);
-    ne = cta_sum<u64>(ne, shu);
+    __shared__ u64 shc[kThreads / 32];
+    u64 cnt = (nb << 48) | ne;
+    cta_sum_pair<kF>(fs, is, cnt, shd, shu, shc);
     const unsigned grid = gridDim.x;
     if (grid == 1) {
-        if (threadIdx.x == 0) norm_write(out, kF, take_sqrt, true, fs, is, nb, ne);
+        if (threadIdx.x == 0) norm_write(out, kF, take_sqrt, true, fs, is, cnt >> 48, cnt & kElemMask);
         return;
     }
     if (threadIdx.x == 0) {
         u64 v = is;
         if (kF) v = fs != fs ? 0x7ff8000000000000ull : (u64)__double_as_longlong(fs);  // never the empty pattern
         *reinterpret_cast<volatile u64 *>(rs.cta_val + blockIdx.x) = v;
-        *reinterpret_cast<volatile u64 *>(rs.cta_blocks + blockIdx.x) = nb;
-        *reinterpret_cast<volatile u64 *>(rs.cta_elems + blockIdx.x) = ne;
+        *reinterpret_cast<volatile u64 *>(rs.cta_cnt + blockIdx.x) = cnt;
     }
     const unsigned n_watch = norm_watchers(grid);
     if (blockIdx.x < grid - n_watch) return;
@@ -390,14 +413,13 @@ __device__ __forceinline__ void norm_epilogue(double fs, unsigned long long is, 
     fs = 0.0, is = 0, nb = 0, ne = 0;
     constexpr int kAhead = 4;  // slots per thread whose loads are in flight together
     for (unsigned base = lo + threadIdx.x; base < hi; base += kAhead * kThreads) {
-        u64 v[kAhead], b[kAhead], e[kAhead];
+        u64 v[kAhead], c[kAhead];
 #pragma unroll
         for (int j = 0; j < kAhead; ++j) {
             const unsigned i = base + j * kThreads;
             if (i < hi) {
                 v[j] = slot_peek(rs.cta_val + i);
-                b[j] = slot_peek(rs.cta_blocks + i);
-                e[j] = slot_peek(rs.cta_elems + i);
+                c[j] = slot_peek(rs.cta_cnt + i);
             }
         }
 #pragma unroll
@@ -405,12 +427,11 @@ __device__ __forceinline__ void norm_epilogue(double fs, unsigned long long is, 
             const unsigned i = base + j * kThreads;
             if (i < hi) {
                 ok = slot_take(rs.cta_val + i, v[j]) && ok;
-                ok = slot_take(rs.cta_blocks + i, b[j]) && ok;
-                ok = slot_take(rs.cta_elems + i, e[j]) && ok;
+                ok = slot_take(rs.cta_cnt + i, c[j]) && ok;
                 if (kF) fs += __longlong_as_double((long long)v[j]);
                 else is += v[j];
-                nb += b[j];
-                ne += e[j];
+                nb += c[j] >> 48;
+                ne += c[j] & kElemMask;
             }
         }
     }

@@ -12,7 +12,7 @@
 // The regular norm pass keeps one partial sum per CTA of its kernel, a few
 // per-tile sums and ticket counters in memory that the context allocated.  Here
 // that scratch is a fixed array in the library's device image instead, so every
-// GPU that loads the library carries it (about 0.4 MiB) until the process
+// GPU that loads the library carries it (about 0.3 MiB) until the process
 // exits, and the block count is capped at SCAR_STATIC_MAX_BLOCKS.
 #include <cstdint>
 #include <mutex>
@@ -28,8 +28,8 @@ namespace {
 constexpr uint64_t kStaticMaxBlocks = SCAR_STATIC_MAX_BLOCKS;
 // The pass launches at most one CTA per kThreads / 4 blocks (the narrowest group has 4 lanes).
 constexpr uint64_t kStaticMaxCtas = kStaticMaxBlocks / (kThreads / 4) + 1;
-// 8-byte words: three slots per CTA, three per watcher.
-constexpr uint64_t kScratchWords = 3 * kStaticMaxCtas + 3 * kMaxWatchers;
+// 8-byte words: two slots per CTA, three per watcher.
+constexpr uint64_t kScratchWords = 2 * kStaticMaxCtas + 3 * kMaxWatchers;
 // Behind them, a band of words that nothing may write: it is filled with a pattern when the address is looked up
 // and scar_static_debug_check_guard counts the bytes that have changed since.
 constexpr uint64_t kGuardWords = 32;
