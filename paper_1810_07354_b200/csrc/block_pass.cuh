@@ -526,10 +526,18 @@ inline uint64_t recover_max_ctas(uint64_t n_blocks, int group_lanes) {
     return (n_blocks + kThreads / group_lanes - 1) / (kThreads / group_lanes) + 1;
 }
 
+// Short blocks (G < 32) are one batch of loads each, so what a pass over them has in flight is the number of
+// resident warps times one batch.  Four CTAs per SM is what the kernel's 64 registers allow; asking for five or
+// six made the compiler spill and the pass 1.4 to 3 times slower (measured), so four is stated, not raised.
+constexpr int kShortBlockCtasPerSm = 4;
+
 // A block's partial enters the sum as the value a score would store (rounded to float32 for float data), so that
 // the squared perturbation of a lost set is exactly the sum of the scores of its blocks.
-template <typename T, int NORM, int G, bool VEC, bool WRITE>
-__global__ void __launch_bounds__(kThreads)
+// MASK: the lost set is a per-block mask (S.mode == 2); otherwise all blocks or runs of blocks.  A template
+// parameter rather than a branch, so that each kernel holds one copy of the streaming loop: with both forms in one
+// kernel the compiler's schedule of that loop changed from build to build (10 to 20 % on the norm pass).
+template <typename T, int NORM, int G, bool VEC, bool WRITE, bool MASK>
+__global__ void __launch_bounds__(kThreads, (G < 32 ? kShortBlockCtasPerSm : 1))
 k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S, unsigned chunk,
                  const float *__restrict__ weight, NormScratch rs, NormInfoDev *out) {
     using E = Elem<T, NORM>;
@@ -539,7 +547,7 @@ k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S, 
     const int lane = threadIdx.x & (G - 1), gi = threadIdx.x / G;
     double fs = 0.0;
     u64 is = 0, nb = 0, ne = 0;
-    if (S.mode == 2) {
+    if (MASK) {
         // Per-block mask: the CTA takes `chunk` consecutive mask entries, writes the ids of the lost blocks
         // among them, in order, to a list in shared memory, and its groups walk that list side by side, so
         // that every group has a lost block to work on however sparse the mask is.

@@ -516,12 +516,23 @@ template <typename T, int NORM> int launch_recover_as(scar_ctx *c, const LostSet
     dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
         constexpr int G = decltype(gl)::value;
         constexpr bool VEC = decltype(vec)::value;
-        if (write)
-            k_recover_blocks<T, NORM, G, VEC, true><<<sh.grid, kThreads, 0, c->stream>>>(
-                static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, sh.chunk, c->d_weight, c->rs, c->d_norm);
-        else
-            k_recover_blocks<T, NORM, G, VEC, false><<<sh.grid, kThreads, 0, c->stream>>>(
-                static_cast<T *>(c->x), static_cast<const T *>(c->z), c->g, S, sh.chunk, c->d_weight, c->rs, c->d_norm);
+        T *x = static_cast<T *>(c->x);
+        const T *z = static_cast<const T *>(c->z);
+        if (S.mode == 2) {
+            if (write)
+                k_recover_blocks<T, NORM, G, VEC, true, true><<<sh.grid, kThreads, 0, c->stream>>>(
+                    x, z, c->g, S, sh.chunk, c->d_weight, c->rs, c->d_norm);
+            else
+                k_recover_blocks<T, NORM, G, VEC, false, true><<<sh.grid, kThreads, 0, c->stream>>>(
+                    x, z, c->g, S, sh.chunk, c->d_weight, c->rs, c->d_norm);
+        } else {
+            if (write)
+                k_recover_blocks<T, NORM, G, VEC, true, false><<<sh.grid, kThreads, 0, c->stream>>>(
+                    x, z, c->g, S, sh.chunk, c->d_weight, c->rs, c->d_norm);
+            else
+                k_recover_blocks<T, NORM, G, VEC, false, false><<<sh.grid, kThreads, 0, c->stream>>>(
+                    x, z, c->g, S, sh.chunk, c->d_weight, c->rs, c->d_norm);
+        }
     });
     ++c->launches;
     record(c, 4);

@@ -83,9 +83,15 @@ int run_static(const void *d_x, const void *d_z, const Geom &g, const LostSet &S
     T *x = static_cast<T *>(const_cast<void *>(d_x));  // the read-only instantiation never stores
     const T *z = static_cast<const T *>(d_z);
     NormInfoDev *out = reinterpret_cast<NormInfoDev *>(d_out);
-#define SCAR_STATIC_LAUNCH(G_, VEC_)                                                                            \
-    k_recover_blocks<T, kNormDefault, G_, VEC_, false><<<sh.grid, kThreads, 0, stream>>>(x, z, g, S, sh.chunk, \
-                                                                                       nullptr, rs, out)
+#define SCAR_STATIC_LAUNCH(G_, VEC_)                                                                               \
+    do {                                                                                                           \
+        if (S.mode == 2)                                                                                           \
+            k_recover_blocks<T, kNormDefault, G_, VEC_, false, true><<<sh.grid, kThreads, 0, stream>>>(           \
+                x, z, g, S, sh.chunk, nullptr, rs, out);                                                           \
+        else                                                                                                       \
+            k_recover_blocks<T, kNormDefault, G_, VEC_, false, false><<<sh.grid, kThreads, 0, stream>>>(          \
+                x, z, g, S, sh.chunk, nullptr, rs, out);                                                           \
+    } while (0)
     if (g.vec_ok) {
         if (G == 4) SCAR_STATIC_LAUNCH(4, true);
         else if (G == 8) SCAR_STATIC_LAUNCH(8, true);
