@@ -526,10 +526,12 @@ inline uint64_t recover_max_ctas(uint64_t n_blocks, int group_lanes) {
     return (n_blocks + kThreads / group_lanes - 1) / (kThreads / group_lanes) + 1;
 }
 
-// Short blocks (G < 32) are one batch of loads each, so what a pass over them has in flight is the number of
-// resident warps times one batch.  Four CTAs per SM is what the kernel's 64 registers allow; asking for five or
-// six made the compiler spill and the pass 1.4 to 3 times slower (measured), so four is stated, not raised.
-constexpr int kShortBlockCtasPerSm = 4;
+// What a streaming pass has in flight is the number of resident warps times what a warp has in flight, so the
+// kernels are held to the registers that let four CTAs share an SM (64 per thread), except the restoring pass
+// over long blocks, whose hand-pipelined loop keeps two batches per lane in registers and settles for two.
+// Asking for five or six CTAs made the compiler spill and the short-block passes 1.4 to 3 times slower; leaving
+// the bound open let it take 96 registers for the read-only pass and lose a fifth of its speed (both measured).
+constexpr int kStreamCtasPerSm = 4;
 
 // A block's partial enters the sum as the value a score would store (rounded to float32 for float data), so that
 // the squared perturbation of a lost set is exactly the sum of the scores of its blocks.
@@ -537,7 +539,7 @@ constexpr int kShortBlockCtasPerSm = 4;
 // parameter rather than a branch, so that each kernel holds one copy of the streaming loop: with both forms in one
 // kernel the compiler's schedule of that loop changed from build to build (10 to 20 % on the norm pass).
 template <typename T, int NORM, int G, bool VEC, bool WRITE, bool MASK>
-__global__ void __launch_bounds__(kThreads, (G < 32 ? kShortBlockCtasPerSm : 1))
+__global__ void __launch_bounds__(kThreads, (WRITE && G == 32 ? 2 : kStreamCtasPerSm))
 k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S, unsigned chunk,
                  const float *__restrict__ weight, NormScratch rs, NormInfoDev *out) {
     using E = Elem<T, NORM>;
