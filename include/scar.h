@@ -274,9 +274,10 @@ int scar_recover_partial_host(scar_ctx *ctx, void *h_x, const uint8_t *h_lost_sh
  *
  *   drain_init     switches the context to drain mode and allocates the second
  *                  device output set plus two pinned host mirrors.  From then
- *                  on every save is limited to max_k blocks and to
- *                  k * (longest block) <= max_payload_elems elements
- *                  (SCAR_ERR_CAPACITY otherwise, nothing enqueued).  Waits for
+ *                  on every save is limited to max_k blocks and to layouts whose
+ *                  k longest blocks together hold at most max_payload_elems
+ *                  elements (whatever the save then selects fits; otherwise
+ *                  SCAR_ERR_CAPACITY, nothing enqueued).  Waits for
  *                  the context's stream.  Once per context.
  *   drain_enqueue  hands the most recent save (there must be one that was not
  *                  handed over yet: SCAR_ERR_STATE otherwise) to the drain

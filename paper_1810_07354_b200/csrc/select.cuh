@@ -271,9 +271,10 @@ __device__ __forceinline__ unsigned long long boundary_len(const S *__restrict__
     return pl[0];
 }
 
-// REG: every CTA owns exactly one tile and keeps its keys in registers.  never != 0 (self-test only) makes every
-// wait expect one arrival more than there are CTAs, so that it runs out.
-template <typename S, bool REG>
+// The general form: every CTA owns a contiguous range of tiles and re-reads their keys in every phase (used when
+// there are more tiles than SMs; k_select_tile below is the form for one tile per CTA).  never != 0 (self-test
+// only) makes every wait expect one arrival more than there are CTAs, so that it runs out.
+template <typename S>
 __global__ void __launch_bounds__(kSelThreads, 1)
 k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st, SaveInfoDev *info,
          uint32_t *__restrict__ sel, unsigned long long *__restrict__ poff, unsigned n_tiles, unsigned tiles_per_cta,
@@ -299,7 +300,6 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
     const u64 key_or = KT::kSkippable ? st->key_or : ~0ull;  // put back to 0 after the exchange
     K key[kSelPerThread];
     unsigned valid = 0;
-    if (REG) load_keys<S>(score, B, (u64)t_lo * kSelTile + (u64)threadIdx.x * kSelPerThread, key, valid);
     for (int i = threadIdx.x; i < kHistBins; i += kSelThreads) sh_hist[i] = 0;
     if (threadIdx.x == 0) {
         sh_boundary = -1;
@@ -320,7 +320,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
                 continue;
             }
             for (unsigned t = t_lo; t < t_hi; ++t) {
-                if (!REG) load_keys<S>(score, B, (u64)t * kSelTile + (u64)threadIdx.x * kSelPerThread, key, valid);
+                load_keys<S>(score, B, (u64)t * kSelTile + (u64)threadIdx.x * kSelPerThread, key, valid);
 #pragma unroll
                 for (int j = 0; j < kSelPerThread; ++j) {
                     const bool match = p == 0 || ((u64)key[j] >> (shift + width)) == prefix;
@@ -350,7 +350,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
         u64 five[5] = {0, 0, 0, 0, 0};  // c_gt, c_eq, c_nf, len_gt, len_eq
         for (unsigned t = t_lo; t < t_hi; ++t) {
             const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kSelPerThread;
-            if (!REG) load_keys<S>(score, B, first, key, valid);
+            load_keys<S>(score, B, first, key, valid);
 #pragma unroll
             for (int j = 0; j < kSelPerThread; ++j) {
                 if (!(valid >> j & 1u)) continue;
@@ -436,7 +436,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
         u64 run_eq = my_eq_before, pos_base = my_sel_base, off_base = my_len_base;
         for (unsigned t = t_lo; t < t_hi; ++t) {
             const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kSelPerThread;
-            if (!REG) load_keys<S>(score, B, first, key, valid);
+            load_keys<S>(score, B, first, key, valid);
             unsigned gt_bits = 0, eq_bits = 0;
 #pragma unroll
             for (int j = 0; j < kSelPerThread; ++j)
