@@ -258,6 +258,35 @@ def test_more_blocks_than_one_selection_tile_per_cta(kind):
         ck.close()
 
 
+@pytest.mark.parametrize("nb", [20_000, 650_000])
+@pytest.mark.parametrize("kind", ["f32", "i32"])
+def test_ties_run_out_inside_one_cta_with_blocks_of_many_lengths(nb, kind):
+    """Explicit ragged layout (block lengths 0..9, so every offset needs the lengths of what was taken before it),
+    60 % of the blocks unchanged (score exactly 0), and k beyond the changed blocks: the k-th score is 0, the ties
+    go to the lowest ids and run out inside one selection CTA; the CTAs behind it need the summed length of what
+    it takes.  20 000 blocks: five CTAs of the one-tile kernel; 650 000: the several-tiles-per-CTA kernel."""
+    r = rng(31 + nb)
+    lens = r.integers(0, 10, size=nb)
+    boff = np.concatenate([[0], np.cumsum(lens)]).astype(np.uint64)
+    n = int(boff[-1])
+    changed = r.random(nb) < 0.4
+    mask = np.repeat(changed, lens)
+    if kind == "f32":
+        z = r.standard_normal(n).astype(np.float32)
+        x = (z + mask * r.standard_normal(n).astype(np.float32)).astype(np.float32)
+    else:
+        z = r.integers(0, 100, size=n).astype(np.int32)
+        x = (z + mask * r.integers(1, 5, size=n)).astype(np.int32)
+    n_changed = int(((lens > 0) & changed).sum())
+    for k in (n_changed + nb // 5, n_changed + 1, nb - 1):
+        xd = parity.to_dev(x)
+        ck = parity.make_ctx(xd, z, boff=boff, n_shards=4)
+        ora = oracle.priority_save(x, z, boff, k=k)
+        got = parity.check_save(ck, ck.priority_save_k(k), x, z, boff, ora)
+        assert got["exact"], "ties at exactly zero leave no freedom"
+        ck.close()
+
+
 def test_uint64_keys_above_32_bits():
     r = rng(8)
     nb, blk = 4000, 16
@@ -329,7 +358,8 @@ def test_masks_empty_full_and_more_shards_than_blocks():
     ck.close()
 
 
-@pytest.mark.parametrize("n_shards,pattern", [(100, "alternate"), (64, "pairs"), (33, "alternate"), (7, "ends")])
+@pytest.mark.parametrize("n_shards,pattern", [(100, "alternate"), (64, "pairs"), (33, "alternate"), (7, "ends"),
+                                              (3000, "alternate")])  # more shards than travel by value: staged copy
 def test_many_lost_shard_runs(n_shards, pattern):
     # few runs travel inside the launch parameters, many fall back to a device-side block mask
     w = make_workload("tiny", n_elems=1 << 18, block_elems=64)  # 4096 blocks
