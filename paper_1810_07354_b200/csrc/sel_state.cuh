@@ -38,12 +38,14 @@ constexpr int kSelStamps = 32;
     } while (0)
 #endif
 
-// What one CTA tells the others once tau is known.
+// What one CTA tells the others once tau is known.  Every word holds its value PLUS ONE, and the state is zero
+// when a selection starts: a word that reads non-zero has arrived (an aligned word is written whole), so the
+// writer needs no fence and the reader no separate flag; it polls until all the words it needs are there.
 struct SelRecord {
     unsigned c_gt;   // keys > tau
     unsigned c_eq;   // keys == tau
     unsigned c_nf;   // non-finite scores
-    unsigned ready;  // set last
+    unsigned unused;
     unsigned long long len_gt;  // summed block lengths of the keys > tau
     unsigned long long len_eq;
 };

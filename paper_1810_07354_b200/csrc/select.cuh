@@ -110,9 +110,6 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned *p) {
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(__cvta_generic_to_global(p)) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_release(unsigned *p, unsigned v) {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(__cvta_generic_to_global(p)), "r"(v) : "memory");
-}
 
 // Polls *word until it reaches target.  False when the wait was abandoned: after kSpinLimit polls, or as soon
 // as another CTA has recorded an error.
@@ -124,6 +121,43 @@ __device__ __forceinline__ bool spin_until_at_least(const unsigned *word, unsign
         if (tries > 16) __nanosleep(tries > 4096 ? 256 : 32);
     }
     return true;
+}
+
+// Publishes this CTA's record (see SelRecord: value + 1 per word, no fence).
+__device__ __forceinline__ void rec_publish(SelRecord *r, unsigned c_gt, unsigned c_eq, unsigned c_nf,
+                                            unsigned long long len_gt, unsigned long long len_eq) {
+    *reinterpret_cast<volatile unsigned long long *>(&r->len_gt) = len_gt + 1;
+    *reinterpret_cast<volatile unsigned long long *>(&r->len_eq) = len_eq + 1;
+    *reinterpret_cast<volatile unsigned *>(&r->c_gt) = c_gt + 1;
+    *reinterpret_cast<volatile unsigned *>(&r->c_eq) = c_eq + 1;
+    *reinterpret_cast<volatile unsigned *>(&r->c_nf) = c_nf + 1;
+}
+
+// Waits (with the usual bound) until the record of a CTA has arrived and returns its values; the lengths only when
+// asked for.  False when the wait was abandoned.
+__device__ __forceinline__ bool rec_take(const SelRecord *r, bool want_lens, const SelState *st, unsigned &c_gt,
+                                         unsigned &c_eq, unsigned &c_nf, unsigned long long &len_gt,
+                                         unsigned long long &len_eq) {
+    unsigned tries = 0;
+    for (;;) {
+        unsigned x, y, z;  // the fourth word of the vector is padding
+        asm volatile("{ .reg .u32 pad; ld.volatile.global.v4.u32 {%0, %1, %2, pad}, [%3]; }"
+                     : "=r"(x), "=r"(y), "=r"(z)
+                     : "l"(__cvta_generic_to_global(r))
+                     : "memory");
+        unsigned long long lg = 1, le = 1;
+        if (want_lens) {
+            lg = *reinterpret_cast<const volatile unsigned long long *>(&r->len_gt);
+            le = *reinterpret_cast<const volatile unsigned long long *>(&r->len_eq);
+        }
+        if (x && y && z && lg && le) {
+            c_gt = x - 1, c_eq = y - 1, c_nf = z - 1, len_gt = lg - 1, len_eq = le - 1;
+            return true;
+        }
+        ++tries;
+        if (tries > kSpinLimit || ((tries & 255u) == 0 && ld_acquire(&st->error) != 0)) return false;
+        if (tries > 16) __nanosleep(tries > 4096 ? 256 : 32);
+    }
 }
 
 __device__ __forceinline__ void sel_fail(SelState *st, SaveInfoDev *info) {
@@ -370,14 +404,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
         cta_sum_n<5, kSelThreads>(five, sh_red);
         SEL_STAMP(st, 26);  // own counts known
         if (threadIdx.x == 0) {
-            SelRecord *r = &st->rec[blockIdx.x];
-            r->c_gt = (unsigned)five[0];
-            r->c_eq = (unsigned)five[1];
-            r->c_nf = (unsigned)five[2];
-            r->len_gt = five[3];
-            r->len_eq = five[4];
-            __threadfence();
-            st_release(&r->ready, 1u);
+            rec_publish(&st->rec[blockIdx.x], (unsigned)five[0], (unsigned)five[1], (unsigned)five[2], five[3], five[4]);
         }
     }
 
@@ -389,17 +416,10 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
         u64 e = 0, gt = 0, nf = 0, lg = 0, le = 0;
         bool ok = true;
         if (c < gridDim.x + never) {
-            const SelRecord *r = &st->rec[c];
-            ok = spin_until_at_least(&r->ready, 1u, st);
-            if (!ok) {
-                sel_fail(st, info);
-            } else if (c < gridDim.x) {
-                e = __ldcg(&r->c_eq);
-                gt = __ldcg(&r->c_gt);
-                nf = __ldcg(&r->c_nf);
-                lg = __ldcg(&r->len_gt);
-                le = __ldcg(&r->len_eq);
-            }
+            unsigned e32 = 0, gt32 = 0, nf32 = 0;
+            ok = rec_take(&st->rec[c], true, st, gt32, e32, nf32, lg, le);
+            e = e32, gt = gt32, nf = nf32;
+            if (!ok) sel_fail(st, info);
         }
         alive = __syncthreads_and(ok) != 0;
         SEL_STAMP(st, 27);  // every CTA's record read
@@ -503,34 +523,84 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
 // unrolled, which keeps the code short; counts travel as 32-bit words and are added with the warp-reduce
 // instruction; one packed scan over the CTAs' records gives all prefix sums; and layouts whose blocks all have
 // one length skip every sum of lengths.
+//
+// A digit pass needs no arrival counter here.  Every CTA knows how many keys take part in the pass (all of them in
+// the first, afterwards the count of the bin resolved before), and the global histogram only grows: a CTA re-reads
+// the histogram until its bins add up to that number, and then every bin it read has its final value.  The
+// reading that finds the histogram complete is also the one the digit is resolved from, so the wait costs no
+// fence, no atomic with a dependent poll and no second read.  expected + 1 can never be reached (self-test).
+constexpr unsigned kHistPollLimit = 1u << 19;  // polls of about half a microsecond each, sleeping 64 ns between them
+
 template <int WIDTH>
-__device__ __forceinline__ unsigned resolve_digit32_w(const unsigned *hist, unsigned &remaining, unsigned *sh_scan,
-                                                      unsigned *sh_out) {
+__device__ __forceinline__ bool resolve_digit_when_complete(const unsigned *hist, unsigned expected, unsigned &remaining,
+                                                            unsigned &digit, unsigned &bin_count, const SelState *st,
+                                                            unsigned (*sh_w)[kSelThreads / 32], unsigned *sh_out,
+                                                            int *sh_stop) {
     constexpr int nb = 1 << WIDTH;
     constexpr int per = nb / kSelThreads;  // 4 or 2 consecutive bins per thread, highest bins in thread 0
-    unsigned local[4] = {0, 0, 0, 0};
+    constexpr int kWarps = kSelThreads / 32;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const unsigned *src = hist + (nb - (int)(threadIdx.x + 1) * per);
-    if (per == 4) {
-        const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(src));
-        local[0] = v.w, local[1] = v.z, local[2] = v.y, local[3] = v.x;
-    } else {
-        const uint2 v = __ldcg(reinterpret_cast<const uint2 *>(src));
-        local[0] = v.y, local[1] = v.x;
-    }
-    const unsigned sum = (local[0] + local[1]) + (local[2] + local[3]);
-    unsigned cum = cta_excl_scan<unsigned, kSelThreads>(sum, sh_scan, nullptr);
-#pragma unroll
-    for (int i = 0; i < per; ++i) {
-        const unsigned h = local[i];
-        if (cum < remaining && remaining <= cum + h) {
-            sh_out[0] = (unsigned)(nb - 1 - ((int)threadIdx.x * per + i));
-            sh_out[1] = remaining - cum;
+    unsigned local[4] = {0, 0, 0, 0};
+    unsigned sum = 0;
+    for (unsigned iter = 0;; ++iter) {
+        if (per == 4) {
+            unsigned a, b, c, d;
+            asm volatile("ld.volatile.global.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(a), "=r"(b), "=r"(c), "=r"(d)
+                         : "l"(__cvta_generic_to_global(src))
+                         : "memory");
+            local[0] = d, local[1] = c, local[2] = b, local[3] = a;
+        } else {
+            unsigned a, b;
+            asm volatile("ld.volatile.global.v2.u32 {%0, %1}, [%2];"
+                         : "=r"(a), "=r"(b)
+                         : "l"(__cvta_generic_to_global(src))
+                         : "memory");
+            local[0] = b, local[1] = a;
         }
-        cum += h;
+        sum = (local[0] + local[1]) + (local[2] + local[3]);
+        const unsigned wsum = __reduce_add_sync(0xffffffffu, sum);
+        unsigned *buf = sh_w[iter & 1];  // two buffers: a fast warp may already write the next round's sums
+        if (lane == 0) buf[w] = wsum;
+        if (threadIdx.x == 0)
+            sh_stop[iter & 1] = iter > kHistPollLimit || ((iter & 63u) == 63u && ld_acquire(&st->error) != 0);
+        __syncthreads();
+        unsigned total = 0, before = 0;
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) {
+            const unsigned t = buf[i];
+            if (i < w) before += t;
+            total += t;
+        }
+        if (total == expected) {
+            // exclusive prefix of this thread's bins, highest bins first: warps before, lanes before
+            unsigned inc = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned n = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += n;
+            }
+            unsigned cum = before + inc - sum;
+#pragma unroll
+            for (int i = 0; i < per; ++i) {
+                const unsigned h = local[i];
+                if (cum < remaining && remaining <= cum + h) {
+                    sh_out[0] = (unsigned)(nb - 1 - ((int)threadIdx.x * per + i));
+                    sh_out[1] = remaining - cum;
+                    sh_out[2] = h;
+                }
+                cum += h;
+            }
+            __syncthreads();
+            digit = sh_out[0];
+            remaining = sh_out[1];
+            bin_count = sh_out[2];
+            return true;  // the next write to sh_out / sh_w comes after further barriers
+        }
+        if (sh_stop[iter & 1]) return false;  // two buffers, as for the sums
+        if (iter > 8) __nanosleep(64);
     }
-    __syncthreads();
-    remaining = sh_out[1];
-    return sh_out[0];  // the next write to sh_out comes after further barriers
 }
 
 template <typename S>
@@ -546,14 +616,15 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
     __shared__ K sh_key[kSelThreads * kPad];
     __shared__ unsigned sh_hist[kHistBins];
     __shared__ unsigned sh_scan[kWarps];
+    __shared__ unsigned sh_poll[2][kWarps];
+    __shared__ int sh_stop[2];
     __shared__ u64 sh_scan64[kWarps];
-    __shared__ unsigned sh_out[2];
+    __shared__ unsigned sh_out[3];
     __shared__ unsigned sh_w[kWarps];
     __shared__ u64 sh_wl[2 * kWarps];
     __shared__ u64 sh_mine[3];
     __shared__ int sh_boundary;
     __shared__ unsigned sh_boundary_take;
-    __shared__ int sh_ok;
 
     griddep_launch();  // the pack kernel may be scheduled while this one runs; it waits before reading sel / poff
     SEL_STAMP(st, 0);
@@ -583,7 +654,7 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
 
     // ---- digit passes: tau = the k-th largest key, need = how many keys equal to tau are taken
     u64 prefix = 0;
-    unsigned need = k;
+    unsigned need = k, taking_part = B;  // keys that enter the next histogram: all, then those of the resolved bin
     if (!none) {
         for (int p = 0; p < KT::kPasses && alive; ++p) {
             const int shift = KT::shift(p), width = KT::width(p);
@@ -607,14 +678,19 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
                 }
             }
             SEL_STAMP(st, 3 + 4 * p);  // flushed
-            alive = sel_arrive_wait(&st->arrive[p], gridDim.x + never, st, info, &sh_ok);
-            SEL_STAMP(st, 4 + 4 * p);  // every CTA has arrived
+            SEL_STAMP(st, 4 + 4 * p);
+            unsigned d = 0, h = 0;
+            alive = width == 11 ? resolve_digit_when_complete<11>(st->hist[p], taking_part + never, need, d, h, st, sh_poll,
+                                                                  sh_out, sh_stop)
+                                : resolve_digit_when_complete<10>(st->hist[p], taking_part + never, need, d, h, st, sh_poll,
+                                                                  sh_out, sh_stop);
             if (alive) {
-                const unsigned d = width == 11 ? resolve_digit32_w<11>(st->hist[p], need, sh_scan, sh_out)
-                                               : resolve_digit32_w<10>(st->hist[p], need, sh_scan, sh_out);
                 prefix = (prefix << width) | d;
+                taking_part = h;  // the keys of the resolved bin are the ones the next pass counts
+            } else if (threadIdx.x == 0) {
+                sel_fail(st, info);
             }
-            SEL_STAMP(st, 5 + 4 * p);  // digit resolved
+            SEL_STAMP(st, 5 + 4 * p);  // histogram complete and digit resolved
         }
     }
     const K tau = (K)prefix;
@@ -662,14 +738,7 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
         my_gt = c_gt, my_eq = c_eq;
         SEL_STAMP(st, 26);  // own counts known
         if (threadIdx.x == 0) {
-            SelRecord *r = &st->rec[blockIdx.x];
-            r->c_gt = c_gt;
-            r->c_eq = c_eq;
-            r->c_nf = t_nf;
-            r->len_gt = lgt;
-            r->len_eq = leq;
-            __threadfence();
-            st_release(&r->ready, 1u);
+            rec_publish(&st->rec[blockIdx.x], c_gt, c_eq, t_nf, lgt, leq);
         }
     }
 
@@ -683,18 +752,8 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
         u64 lg = 0, le = 0;
         bool ok = true;
         if (c < gridDim.x + never) {
-            const SelRecord *r = &st->rec[c];
-            ok = spin_until_at_least(&r->ready, 1u, st);
-            if (!ok) {
-                sel_fail(st, info);
-            } else if (c < gridDim.x) {
-                const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(r));
-                gt = v.x, e = v.y, nf = v.z;
-                if (!ulen) {
-                    lg = __ldcg(&r->len_gt);
-                    le = __ldcg(&r->len_eq);
-                }
-            }
+            ok = rec_take(&st->rec[c], !ulen, st, gt, e, nf, lg, le);
+            if (!ok) sel_fail(st, info);
         }
         alive = __syncthreads_and(ok) != 0;
         SEL_STAMP(st, 27);  // every CTA's record read
