@@ -23,6 +23,7 @@ constexpr int kMaxSelCtas = kSelThreads;  // the exchange reads one record per t
 // A wait polls at most this often, sleeping 256 ns between polls once it has polled 4096 times: it gives up after
 // a quarter of a second at the earliest and about a second in practice.
 constexpr unsigned kSpinLimit = 1u << 20;
+constexpr unsigned kSelDirectKeys = 64;  // a digit pass over at most this many keys skips the shared histogram
 
 // Diagnostic builds (-DSCAR_SELECT_STAMPS) record where the selection kernel's time goes: thread 0 of CTA 0
 // writes its SM's cycle counter at up to kSelStamps marked points; scar_ckpt_debug_select_stamps reads them.

@@ -614,7 +614,7 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
     constexpr int P = kSelPerThread, kPad = P + 1;  // odd stride: the threads of a warp hit 32 different banks
     constexpr int kWarps = kSelThreads / 32;
     __shared__ K sh_key[kSelThreads * kPad];
-    __shared__ unsigned sh_hist[kHistBins];
+    __shared__ __align__(8) unsigned sh_hist[kHistBins];
     __shared__ unsigned sh_scan[kWarps];
     __shared__ unsigned sh_poll[2][kWarps];
     __shared__ int sh_stop[2];
@@ -643,6 +643,20 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
 #pragma unroll
         for (int j = 0; j < P; ++j) my[j] = key[j];
     }
+    // Rows that end in a shorter block give an implicit layout two block lengths.  Which of this thread's blocks
+    // are the short ones is worked out once; every sum of lengths is then two population counts.
+    const bool two_len = !ulen && !g.boff;
+    const u64 len_full = g.block_elems;
+    u64 len_short = 0;
+    unsigned short_bits = 0;
+    if (two_len) {
+        len_short = g.row_len - (u64)(g.blocks_per_row - 1) * g.block_elems;
+        unsigned j = first % g.blocks_per_row;
+        for (int i = 0; i < P; ++i) {
+            if (j == g.blocks_per_row - 1) short_bits |= 1u << i;
+            if (++j == g.blocks_per_row) j = 0;
+        }
+    }
     for (int i = threadIdx.x; i < kHistBins; i += kSelThreads) sh_hist[i] = 0;
     if (threadIdx.x == 0) {
         sh_boundary = -1;
@@ -663,19 +677,35 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
                 prefix <<= width;
                 continue;
             }
+            // A handful of keys left (the usual state of the last pass) go to the global histogram one by one: the
+            // shared histogram, its barrier and the sweep over its bins would cost more.  taking_part is the same
+            // number in every CTA, so all of them take the same branch.
+            const bool direct = p != 0 && taking_part <= kSelDirectKeys;
 #pragma unroll 2
             for (int j = 0; j < nv; ++j) {
                 const u64 key = my[j];
-                if (p == 0 || (key >> (shift + width)) == prefix) atomicAdd(&sh_hist[(unsigned)((key >> shift) & mask)], 1u);
-            }
-            __syncthreads();
-            SEL_STAMP(st, 2 + 4 * p);  // pass p: shared histogram built
-            for (int i = threadIdx.x; i < (1 << width); i += kSelThreads) {
-                const unsigned c = sh_hist[i];
-                if (c) {
-                    atomicAdd(&st->hist[p][i], c);
-                    sh_hist[i] = 0;  // ready for the next pass
+                if (p == 0 || (key >> (shift + width)) == prefix) {
+                    const unsigned bin = (unsigned)((key >> shift) & mask);
+                    if (direct) atomicAdd(&st->hist[p][bin], 1u);  // two atomics, not one through a generic pointer
+                    else atomicAdd(&sh_hist[bin], 1u);
                 }
+            }
+            if (!direct) {
+                __syncthreads();
+                SEL_STAMP(st, 2 + 4 * p);  // pass p: shared histogram built
+                // two neighbouring bins per reduction (a count never carries into its neighbour: a histogram holds
+                // fewer than 2^32 keys): half as many updates meet in L2
+                u64 *pairs = reinterpret_cast<u64 *>(st->hist[p]);
+                uint2 *mine = reinterpret_cast<uint2 *>(sh_hist);
+                for (int i = threadIdx.x; i < (1 << (width - 1)); i += kSelThreads) {
+                    const uint2 c = mine[i];
+                    if (c.x | c.y) {
+                        atomicAdd(&pairs[i], (u64)c.x | ((u64)c.y << 32));
+                        mine[i] = make_uint2(0u, 0u);  // ready for the next pass
+                    }
+                }
+            } else {
+                SEL_STAMP(st, 2 + 4 * p);
             }
             SEL_STAMP(st, 3 + 4 * p);  // flushed
             SEL_STAMP(st, 4 + 4 * p);
@@ -710,7 +740,13 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
         // per warp at most 256 of each: three 10-bit fields in one word, one warp-reduce instruction
         const unsigned packed = __reduce_add_sync(0xffffffffu, __popc(gt_bits) | (__popc(eq_bits) << 10) | (c_nf << 20));
         u64 lgt = 0, leq = 0;
-        if (!ulen) {
+        if (two_len) {
+            const unsigned shorts = __reduce_add_sync(0xffffffffu, __popc(gt_bits & short_bits) |
+                                                                       (__popc(eq_bits & short_bits) << 10));
+            const unsigned s_gt = shorts & 1023u, s_eq = shorts >> 10;
+            lgt = (u64)((packed & 1023u) - s_gt) * len_full + (u64)s_gt * len_short;
+            leq = (u64)(((packed >> 10) & 1023u) - s_eq) * len_full + (u64)s_eq * len_short;
+        } else if (!ulen) {
             BlockLens bl(g, first);
             for (int j = 0; j < nv; ++j) {
                 const u64 len = bl.next();
@@ -831,24 +867,38 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
                 }
         } else {
             u64 lsum = 0;
-            BlockLens bl(g, first);
-            for (int j = 0; j < nv; ++j) {
-                const u64 len = bl.next();
-                if (take_bits >> j & 1u) lsum += len;
+            if (two_len) {
+                lsum = (u64)__popc(take_bits & ~short_bits) * len_full + (u64)__popc(take_bits & short_bits) * len_short;
+            } else {
+                BlockLens bl(g, first);
+                for (int j = 0; j < nv; ++j) {
+                    const u64 len = bl.next();
+                    if (take_bits >> j & 1u) lsum += len;
+                }
             }
             // one scan for both outputs: block counts in the top 16 bits (at most 4096 per tile), summed
             // lengths below (a buffer has fewer than 2^48 elements: init rejects more)
             const u64 both = cta_excl_scan<u64, kSelThreads>(((u64)__popc(take_bits) << 48) | lsum, sh_scan64, nullptr);
             unsigned pos = my_sel_base + (unsigned)(both >> 48);
             u64 off = my_len_base + (both & ((1ull << 48) - 1));
-            BlockLens bl2(g, first);
-            for (int j = 0; j < nv; ++j) {
-                const u64 len = bl2.next();
-                if (take_bits >> j & 1u) {
-                    sel[pos] = first + j;
-                    poff[pos] = off;
-                    ++pos;
-                    off += len;
+            if (two_len) {
+                for (int j = 0; j < nv; ++j)
+                    if (take_bits >> j & 1u) {
+                        sel[pos] = first + j;
+                        poff[pos] = off;
+                        ++pos;
+                        off += (short_bits >> j & 1u) ? len_short : len_full;
+                    }
+            } else {
+                BlockLens bl(g, first);
+                for (int j = 0; j < nv; ++j) {
+                    const u64 len = bl.next();
+                    if (take_bits >> j & 1u) {
+                        sel[pos] = first + j;
+                        poff[pos] = off;
+                        ++pos;
+                        off += len;
+                    }
                 }
             }
         }
