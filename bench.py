@@ -442,6 +442,28 @@ def measure_workload(api, name, n_elems, rank, dev, steps, warmup, barrier):
     return m
 
 
+def event_floor(dev, reps=50):
+    """What a pair of CUDA events reads around a kernel that does nothing: a one-element fill launched behind a
+    kernel that is still running, as every timed phase is.  The phase times of the small parameter sets (the
+    selection above all) contain this much that is not the kernel."""
+    import torch
+
+    one = torch.zeros(1, device=dev)
+    busy = torch.zeros(1 << 24, device=dev)
+    ts = []
+    for _ in range(reps + 5):
+        busy.add_(1.0)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        one.zero_()
+        b.record()
+        b.synchronize()
+        ts.append(a.elapsed_time(b))
+    ts = ts[5:]
+    return {"ms": float(np.median(ts)), "ms_min": float(np.min(ts)),
+            "what": "a one-element fill between two events, behind a running kernel"}
+
+
 def summarise(m, peak):
     """Per-r save figures, norm and recovery figures of one measured workload."""
     scanned = 2 * m.n * ELEM
@@ -529,6 +551,7 @@ def run_gpu(args):
                      "traffic": recorded_traffic(n) if args.workload == "cnn" else None,
                      "bytes_per_launch": scanned, "ms_per_launch": m.score_ms},
         "gpu_launches": int(m.launches),
+        "event_floor": event_floor(dev),
         "clocks": clocks,
         "wall_s_timed_region": m.w1 - m.w0,
     }

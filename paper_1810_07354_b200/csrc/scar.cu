@@ -394,12 +394,16 @@ int launch_select(scar_ctx *c, const S *score, const Geom &g, uint64_t k, const 
     unsigned k32 = (unsigned)k, nt = sh.n_tiles, per = sh.tiles_per_cta, never = c->arm_never ? 1u : 0u;
     c->arm_never = false;
     if (per == 1 && sh.grid == 1) {
-        // a single CTA has nobody to wait for: no co-residency to guarantee, and a plain launch starts sooner
-        k_select_tile<S><<<1, kSelThreads, 0, c->stream>>>(score, geom, k32, c->st, out.info, out.sel, out.poff, never);
+        // A single CTA has nobody to wait for: no co-residency to guarantee, a plain launch starts sooner, and its
+        // histograms never leave shared memory.  (The timeout self-test needs a wait, so it runs the form that has one.)
+        if (never)
+            k_select_tile<S, false><<<1, kSelThreads, 0, c->stream>>>(score, geom, k32, c->st, out.info, out.sel, out.poff, never);
+        else
+            k_select_tile<S, true><<<1, kSelThreads, 0, c->stream>>>(score, geom, k32, c->st, out.info, out.sel, out.poff, never);
         CU_TRY(cudaGetLastError());
     } else if (per == 1) {  // the usual case: one tile per CTA
         void *args[] = {&score, &geom, &k32, &c->st, &out.info, &out.sel, &out.poff, &never};
-        CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select_tile<S>), dim3(sh.grid),
+        CU_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&k_select_tile<S, false>), dim3(sh.grid),
                                            dim3(kSelThreads), args, 0, c->stream));
     } else {
         void *args[] = {&score, &geom, &kk, &c->st, &out.info, &out.sel, &out.poff, &nt, &per, &never};
@@ -415,7 +419,7 @@ template <typename S> int select_occupancy(int &occ) {
     int o = 0;
     CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, k_select<S>, kSelThreads, 0));
     occ = o < occ ? o : occ;
-    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, k_select_tile<S>, kSelThreads, 0));
+    CU_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, k_select_tile<S, false>, kSelThreads, 0));
     occ = o < occ ? o : occ;
     return SCAR_OK;
 }

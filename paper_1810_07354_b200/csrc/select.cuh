@@ -141,7 +141,7 @@ __device__ __forceinline__ bool rec_take(const SelRecord *r, bool want_lens, con
     unsigned tries = 0;
     for (;;) {
         unsigned x, y, z;  // the fourth word of the vector is padding
-        asm volatile("{ .reg .u32 pad; ld.volatile.global.v4.u32 {%0, %1, %2, pad}, [%3]; }"
+        asm volatile("{ .reg .u32 pad; ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, pad}, [%3]; }"
                      : "=r"(x), "=r"(y), "=r"(z)
                      : "l"(__cvta_generic_to_global(r))
                      : "memory");
@@ -531,8 +531,11 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
 // fence, no atomic with a dependent poll and no second read.  expected + 1 can never be reached (self-test).
 constexpr unsigned kHistPollLimit = 1u << 19;  // polls of about half a microsecond each, sleeping 64 ns between them
 
-template <int WIDTH>
-__device__ __forceinline__ bool resolve_digit_when_complete(const unsigned *hist, unsigned expected, unsigned &remaining,
+//
+// LOCAL: the histogram is the CTA's own, in shared memory and already complete (a selection that one CTA does
+// alone); the first reading resolves the digit, and the bins are put back to zero for the next pass.
+template <int WIDTH, bool LOCAL>
+__device__ __forceinline__ bool resolve_digit_when_complete(unsigned *hist, unsigned expected, unsigned &remaining,
                                                             unsigned &digit, unsigned &bin_count, const SelState *st,
                                                             unsigned (*sh_w)[kSelThreads / 32], unsigned *sh_out,
                                                             int *sh_stop) {
@@ -540,20 +543,30 @@ __device__ __forceinline__ bool resolve_digit_when_complete(const unsigned *hist
     constexpr int per = nb / kSelThreads;  // 4 or 2 consecutive bins per thread, highest bins in thread 0
     constexpr int kWarps = kSelThreads / 32;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const unsigned *src = hist + (nb - (int)(threadIdx.x + 1) * per);
+    unsigned *src = hist + (nb - (int)(threadIdx.x + 1) * per);
     unsigned local[4] = {0, 0, 0, 0};
     unsigned sum = 0;
     for (unsigned iter = 0;; ++iter) {
-        if (per == 4) {
+        if (LOCAL) {
+            if (per == 4) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(src);
+                local[0] = v.w, local[1] = v.z, local[2] = v.y, local[3] = v.x;
+                *reinterpret_cast<uint4 *>(src) = make_uint4(0u, 0u, 0u, 0u);
+            } else {
+                const uint2 v = *reinterpret_cast<const uint2 *>(src);
+                local[0] = v.y, local[1] = v.x;
+                *reinterpret_cast<uint2 *>(src) = make_uint2(0u, 0u);
+            }
+        } else if (per == 4) {
             unsigned a, b, c, d;
-            asm volatile("ld.volatile.global.v4.u32 {%0, %1, %2, %3}, [%4];"
+            asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];"
                          : "=r"(a), "=r"(b), "=r"(c), "=r"(d)
                          : "l"(__cvta_generic_to_global(src))
                          : "memory");
             local[0] = d, local[1] = c, local[2] = b, local[3] = a;
         } else {
             unsigned a, b;
-            asm volatile("ld.volatile.global.v2.u32 {%0, %1}, [%2];"
+            asm volatile("ld.relaxed.gpu.global.v2.u32 {%0, %1}, [%2];"
                          : "=r"(a), "=r"(b)
                          : "l"(__cvta_generic_to_global(src))
                          : "memory");
@@ -603,7 +616,9 @@ __device__ __forceinline__ bool resolve_digit_when_complete(const unsigned *hist
     }
 }
 
-template <typename S>
+// SOLO: the whole selection is this one CTA's (at most kSelTile blocks): histograms stay in shared memory and
+// nothing is exchanged through global memory.
+template <typename S, bool SOLO>
 __global__ void __launch_bounds__(kSelThreads, 1)
 k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, SaveInfoDev *info,
               uint32_t *__restrict__ sel, unsigned long long *__restrict__ poff, unsigned never) {
@@ -614,7 +629,7 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
     constexpr int P = kSelPerThread, kPad = P + 1;  // odd stride: the threads of a warp hit 32 different banks
     constexpr int kWarps = kSelThreads / 32;
     __shared__ K sh_key[kSelThreads * kPad];
-    __shared__ __align__(8) unsigned sh_hist[kHistBins];
+    __shared__ __align__(16) unsigned sh_hist[kHistBins];
     __shared__ unsigned sh_scan[kWarps];
     __shared__ unsigned sh_poll[2][kWarps];
     __shared__ int sh_stop[2];
@@ -680,7 +695,7 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
             // A handful of keys left (the usual state of the last pass) go to the global histogram one by one: the
             // shared histogram, its barrier and the sweep over its bins would cost more.  taking_part is the same
             // number in every CTA, so all of them take the same branch.
-            const bool direct = p != 0 && taking_part <= kSelDirectKeys;
+            const bool direct = !SOLO && p != 0 && taking_part <= kSelDirectKeys;
 #pragma unroll 2
             for (int j = 0; j < nv; ++j) {
                 const u64 key = my[j];
@@ -690,9 +705,9 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
                     else atomicAdd(&sh_hist[bin], 1u);
                 }
             }
-            if (!direct) {
-                __syncthreads();
-                SEL_STAMP(st, 2 + 4 * p);  // pass p: shared histogram built
+            if (!direct) __syncthreads();
+            SEL_STAMP(st, 2 + 4 * p);  // pass p: histogram built
+            if (!direct && !SOLO) {
                 // two neighbouring bins per reduction (a count never carries into its neighbour: a histogram holds
                 // fewer than 2^32 keys): half as many updates meet in L2
                 u64 *pairs = reinterpret_cast<u64 *>(st->hist[p]);
@@ -704,16 +719,15 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
                         mine[i] = make_uint2(0u, 0u);  // ready for the next pass
                     }
                 }
-            } else {
-                SEL_STAMP(st, 2 + 4 * p);
             }
             SEL_STAMP(st, 3 + 4 * p);  // flushed
             SEL_STAMP(st, 4 + 4 * p);
             unsigned d = 0, h = 0;
-            alive = width == 11 ? resolve_digit_when_complete<11>(st->hist[p], taking_part + never, need, d, h, st, sh_poll,
-                                                                  sh_out, sh_stop)
-                                : resolve_digit_when_complete<10>(st->hist[p], taking_part + never, need, d, h, st, sh_poll,
-                                                                  sh_out, sh_stop);
+            unsigned *hist = SOLO ? sh_hist : st->hist[p];
+            const unsigned expected = SOLO ? taking_part : taking_part + never;
+            alive = width == 11
+                        ? resolve_digit_when_complete<11, SOLO>(hist, expected, need, d, h, st, sh_poll, sh_out, sh_stop)
+                        : resolve_digit_when_complete<10, SOLO>(hist, expected, need, d, h, st, sh_poll, sh_out, sh_stop);
             if (alive) {
                 prefix = (prefix << width) | d;
                 taking_part = h;  // the keys of the resolved bin are the ones the next pass counts
@@ -726,7 +740,8 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
     const K tau = (K)prefix;
 
     // ---- this CTA's record
-    unsigned gt_bits = 0, eq_bits = 0, my_gt = 0, my_eq = 0;
+    unsigned gt_bits = 0, eq_bits = 0, my_gt = 0, my_eq = 0, my_nf = 0;
+    u64 my_lgt = 0, my_leq = 0;
     if (alive) {
         unsigned c_nf = 0;
 #pragma unroll 2
@@ -771,11 +786,9 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
         }
         if (!ulen)
             for (int w = 0; w < kWarps; ++w) lgt += sh_wl[2 * w], leq += sh_wl[2 * w + 1];
-        my_gt = c_gt, my_eq = c_eq;
+        my_gt = c_gt, my_eq = c_eq, my_nf = t_nf, my_lgt = lgt, my_leq = leq;
         SEL_STAMP(st, 26);  // own counts known
-        if (threadIdx.x == 0) {
-            rec_publish(&st->rec[blockIdx.x], c_gt, c_eq, t_nf, lgt, leq);
-        }
+        if (!SOLO && threadIdx.x == 0) rec_publish(&st->rec[blockIdx.x], c_gt, c_eq, t_nf, lgt, leq);
     }
 
     // ---- exchange: thread c takes the record of CTA c; one packed scan gives every prefix sum
@@ -787,7 +800,9 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
         unsigned e = 0, gt = 0, nf = 0;
         u64 lg = 0, le = 0;
         bool ok = true;
-        if (c < gridDim.x + never) {
+        if (SOLO) {
+            if (c == 0) gt = my_gt, e = my_eq, nf = my_nf, lg = my_lgt, le = my_leq;
+        } else if (c < gridDim.x + never) {
             ok = rec_take(&st->rec[c], !ulen, st, gt, e, nf, lg, le);
             if (!ok) sel_fail(st, info);
         }
