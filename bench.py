@@ -736,7 +736,7 @@ def run_select_stamps(args):
         for p in range(6):
             if st[2 + 4 * p] > st[0]:  # this digit pass ran
                 rec[f"pass{p}"] = {"histogram": us(last, 2 + 4 * p), "flush": us(2 + 4 * p, 3 + 4 * p),
-                                   "wait": us(3 + 4 * p, 4 + 4 * p), "resolve": us(4 + 4 * p, 5 + 4 * p)}
+                                   "complete_and_resolved": us(3 + 4 * p, 5 + 4 * p)}
                 last = 5 + 4 * p
         rec.update(counts=us(last, 26), exchange=us(26, 27), scan=us(27, 28), emit=us(28, 29), total=us(0, 29))
         out["per_r"][str(r)] = rec

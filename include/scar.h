@@ -382,10 +382,11 @@ double scar_irreducible_error(double delta_max, double c);
 
 /* Self-test hook for the bounded device-side wait.  The selection kernel's
  * CTAs meet at a few points whose wait gives up after a fixed number of polls
- * (2^20: a quarter of a second at the earliest, about a second in practice)
- * instead of hanging.  This call makes the NEXT prioritized or random save
- * expect one arrival more than its selection has CTAs (host state only), so
- * that its first wait can never complete: that save takes about a second,
+ * (2^19 to 2^20: a quarter of a second at the earliest, about a second in
+ * practice) instead of hanging.  This call makes the NEXT prioritized or
+ * random save wait for one key, one record or one arrival more than its
+ * selection has (host state only), so that its first wait can never
+ * complete: that save takes up to about a second,
  * selects and copies nothing, leaves z untouched, and returns SCAR_ERR_TIMEOUT
  * from the call that reads its result (the save itself with a non-NULL out, or
  * scar_ckpt_last_info).  The save after that one works normally.
@@ -413,8 +414,11 @@ int scar_static_debug_check_guard(uint64_t *bad_bytes);
  * SCAR_ERR_STATE).  Waits for the stream and copies the 32 time stamps of the
  * most recent selection kernel: SM clock cycles of its first CTA at
  *   [0] start, [1] keys loaded, then for digit pass p = 0..5
- *   [2+4p] shared histogram built, [3+4p] flushed to the global histogram,
- *   [4+4p] every CTA has arrived, [5+4p] digit resolved,
+ *   [2+4p] shared histogram built, [3+4p] flushed to the global histogram
+ *   (a selection that one CTA does alone flushes nothing), [4+4p] every CTA
+ *   has arrived (only selections with several tiles per CTA meet at a
+ *   counter; otherwise the same point as [3+4p]), [5+4p] global histogram
+ *   complete and digit resolved,
  *   [26] own counts known, [27] every CTA's record read, [28] output bases
  *   known, [29] ids and offsets written.
  * Stamps of passes that did not run keep the value of an earlier selection (or

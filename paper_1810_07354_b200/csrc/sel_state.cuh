@@ -55,7 +55,7 @@ struct SelState {
     unsigned long long key_or;  // OR of all uint64 keys seen since the last selection
     unsigned long long reserved;
     // ---- everything from here on is zero when a selection starts
-    unsigned arrive[kMaxPasses];  // arrivals after each digit pass
+    unsigned arrive[kMaxPasses];  // arrivals after each digit pass (k_select only; k_select_tile needs none)
     unsigned error;               // non-zero once a wait gave up
     unsigned reserved2;
     unsigned hist[kMaxPasses][kHistBins];

@@ -8,38 +8,38 @@
 // non-negative float32 score (NaN and +Inf both map to the +Inf pattern, so
 // such blocks rank first), or the uint64 l1 score itself.
 //
-// The whole selection is ONE kernel, launched cooperatively (every CTA is
-// resident), because the score array is small (4-8 bytes per block) and a
-// chain of dependent launches costs more than the work itself.  Each CTA owns
-// a contiguous range of 4096-key tiles; when that range is a single tile (up
-// to about 600 000 blocks on a 148-SM device) its keys stay in registers from
-// the first load to the last store.  The CTAs meet at few points, and at each
-// of them a CTA pays for as few dependent trips to the L2 cache as possible:
+// The whole selection is ONE kernel, because the score array is small (4-8 bytes per block) and a chain of
+// dependent launches costs more than the work itself.  Each CTA owns a contiguous range of 4096-key tiles.
+// Three forms:
+//   k_select_tile<S, true>    at most one tile in all: a single CTA, launched plainly, whose histograms never
+//                             leave shared memory
+//   k_select_tile<S, false>   one tile per CTA (up to about 600 000 blocks on a 148-SM device), launched
+//                             cooperatively so that every CTA is resident; keys are loaded once and stay in
+//                             shared memory
+//   k_select<S>               several tiles per CTA, also cooperative; keys are re-read from the score array
+// The CTAs meet at few points, and at each of them a CTA pays for as few dependent trips to the L2 cache as
+// possible:
 //
-//   digit passes   most-significant digit first: shared-memory histogram of
-//                  the keys that match the prefix so far, flushed with integer
-//                  atomics; one arrival counter per pass (fire-and-forget
-//                  increment, then an acquiring poll); every CTA resolves the
-//                  digit from the global histogram (the same small scan in
-//                  every CTA).  Digits that are zero in every uint64 key are
-//                  skipped.
-//   exchange       with the threshold key tau and `need` (how many keys equal
-//                  to tau are taken) every CTA publishes one record: how many
-//                  of its keys lie above / at tau and their summed lengths.
-//                  Thread c of every CTA waits for the record of CTA c, and a
-//                  CTA-wide scan of the records gives the CTA its output bases
-//                  and the totals.  This one step stands for a barrier, the
-//                  per-CTA counts and their prefix sums.
-//   boundary       only when the tau-keys run out inside one CTA's range and
-//                  block lengths differ: the CTAs after it recompute, from that
-//                  CTA's keys, the summed length of the tau-blocks it takes
+//   digit passes   most-significant digit first: shared-memory histogram of the keys that match the prefix so
+//                  far, flushed with integer reductions; every CTA resolves the digit from the global
+//                  histogram (the same small scan in every CTA).  k_select_tile knows how many keys a pass
+//                  counts and simply re-reads the histogram until its bins add up to that number; k_select
+//                  meets at one arrival counter per pass (fire-and-forget increment, then an acquiring poll).
+//                  Digits that are zero in every uint64 key are skipped.
+//   exchange       with the threshold key tau and `need` (how many keys equal to tau are taken) every CTA
+//                  publishes one record: how many of its keys lie above / at tau and their summed lengths.
+//                  A record's words hold value + 1, so a word that reads non-zero has arrived: no fence, no
+//                  flag.  Thread c of every CTA waits for the record of CTA c, and a CTA-wide scan of the
+//                  records gives the CTA its output bases and the totals.  This one step stands for a
+//                  barrier, the per-CTA counts and their prefix sums.
+//   boundary       only when the tau-keys run out inside one CTA's range and block lengths differ: the CTAs
+//                  after it recompute, from that CTA's keys, the summed length of the tau-blocks it takes
 //   emit           ordered compaction into sel[] / poff[]
 //
-// Every wait is bounded: a CTA that gives up records an error and leaves, the
-// others see it and leave too, and the host reports SCAR_ERR_TIMEOUT.  The
-// counters, histograms and records must be zero when the kernel starts
-// (sel_state_clear, run by the kernel that precedes it on the stream, or a
-// memset); the kernel never has to put them back.
+// Every wait is bounded: a CTA that gives up records an error and leaves, the others see it and leave too, and
+// the host reports SCAR_ERR_TIMEOUT.  The counters, histograms and records must be zero when the kernel starts
+// (sel_state_clear, run by the kernel that precedes it on the stream, or a memset); the kernel never has to put
+// them back.
 #pragma once
 #include "block_pass.cuh"
 #include "sel_state.cuh"

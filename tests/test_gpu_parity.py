@@ -520,8 +520,8 @@ def test_empty_buffer():
 @pytest.mark.parametrize("kind", ["f32", "i32"])
 def test_a_barrier_that_cannot_complete_times_out_and_the_context_survives(kind):
     """The selection's grid barrier gives up after a bounded number of tries: the save reports a timeout, has
-    copied nothing, and the next save is exact again.  The wait is made to run out by mis-setting the arrival
-    counter (a flag that nothing sets), never by a fault."""
+    copied nothing, and the next save is exact again.  The wait is made to run out by mis-setting what it
+    waits for (one key more than exists: a condition that nothing fulfils), never by a fault."""
     w = make_workload("tiny", n_elems=1 << 20) if kind == "f32" else make_workload("lda", vocab=20_000, topics=100)
     boff = block_offsets(w.geom)
     xd = parity.to_dev(w.x)
