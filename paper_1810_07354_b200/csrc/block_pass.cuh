@@ -504,19 +504,26 @@ __device__ __forceinline__ W cta_excl_scan(W v, W *sh /*NT/32*/, W *total) {
 // Launch shape of the pass: one group of lanes per lost block; a per-block mask is cut into chunks of `chunk`
 // mask entries (a multiple of kThreads), one CTA each.
 constexpr unsigned kMaxMaskChunk = 4 * kThreads;
+constexpr uint64_t kTwoRoundsFrom = 4096;  // CTAs a one-round launch would have
 struct RecoverShape {
     unsigned grid;
     unsigned chunk;
 };
-inline RecoverShape recover_shape(int mode, uint64_t n_work, int group_lanes) {
+inline RecoverShape recover_shape(int mode, uint64_t n_work, int group_lanes, bool write) {
     RecoverShape r{1, (unsigned)kThreads};
     uint64_t want;
     if (mode == 2) {
         r.chunk = group_lanes < 32 ? 2 * kThreads : kThreads;  // short blocks: more of them per CTA
         want = (n_work + r.chunk - 1) / r.chunk;
     } else {
+        // One work item per group; two, one after the other, when a read-only pass over short blocks would
+        // otherwise need thousands of CTAs that live for one batch of loads and then pay for the CTA-wide sum
+        // (400-byte rows: 68 us instead of 73 us; four and more lost what two gained, and small launches lost
+        // at any number above one).
         const uint64_t groups = kThreads / group_lanes;
-        want = (n_work + groups - 1) / groups;
+        const bool twice = !write && group_lanes < 32 && n_work >= kTwoRoundsFrom * groups;
+        r.chunk = (unsigned)(groups * (twice ? 2 : 1));
+        want = (n_work + r.chunk - 1) / r.chunk;
     }
     r.grid = (unsigned)(want < 1 ? 1 : want);
     return r;
@@ -584,18 +591,21 @@ k_recover_blocks(T *__restrict__ x, const T *__restrict__ z, Geom g, LostSet S, 
             }
         }
     } else {
-        const uint64_t w = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) / G;
-        uint32_t b = 0;
-        const bool valid = S.block_of(w, b);
-        uint64_t beg = 0, len = 0;
-        if (valid) g.range(b, beg, len);
-        const typename E::wide_t s = block_distance<T, NORM, G, VEC, WRITE>(x, z, beg, len, lane);
-        if (valid && lane == 0) {
-            const typename E::score_t sc = weighted<E>(s, weight, b);
-            if (kF) fs = (double)sc;
-            else is = (u64)sc;
-            nb = 1;
-            ne = len;
+        // chunk work items per CTA: one or two per group (recover_shape)
+        for (unsigned w0 = 0; w0 < chunk; w0 += kGroups) {  // same trip count for every thread of the CTA
+            const uint64_t w = (uint64_t)blockIdx.x * chunk + w0 + gi;
+            uint32_t b = 0;
+            const bool valid = S.block_of(w, b);
+            uint64_t beg = 0, len = 0;
+            if (valid) g.range(b, beg, len);
+            const typename E::wide_t s = block_distance<T, NORM, G, VEC, WRITE>(x, z, beg, len, lane);
+            if (valid && lane == 0) {
+                const typename E::score_t sc = weighted<E>(s, weight, b);
+                if (kF) fs += (double)sc;
+                else is += (u64)sc;
+                ++nb;
+                ne += len;
+            }
         }
     }
     norm_epilogue<T>(fs, is, nb, ne, rs, out, NORM == kNormDefault);

@@ -520,7 +520,7 @@ template <typename T, int NORM> int launch_recover_as(scar_ctx *c, const LostSet
         record(c, 5);
         return SCAR_OK;
     }
-    const RecoverShape sh = recover_shape(S.mode, S.n_work, c->group_lanes);
+    const RecoverShape sh = recover_shape(S.mode, S.n_work, c->group_lanes, write);
     dispatch_group(c->group_lanes, c->g.vec_ok != 0, [&](auto gl, auto vec) {
         constexpr int G = decltype(gl)::value;
         constexpr bool VEC = decltype(vec)::value;

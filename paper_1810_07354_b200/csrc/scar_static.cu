@@ -74,7 +74,7 @@ int run_static(const void *d_x, const void *d_z, const Geom &g, const LostSet &S
     if (g.vec_ok) units /= 4.0;
     int G = 4;
     while (G < 32 && G * 4 < units) G <<= 1;
-    const RecoverShape sh = recover_shape(S.mode, S.n_work, G);
+    const RecoverShape sh = recover_shape(S.mode, S.n_work, G, false);
     if (sh.grid > kStaticMaxCtas) return SCAR_ERR_CAPACITY;
     const NormScratch rs = norm_scratch_at(scratch, sh.grid);
     // Every call shares the array, and an earlier call may have laid it out for another grid size: the slots

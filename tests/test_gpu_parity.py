@@ -287,6 +287,37 @@ def test_ties_run_out_inside_one_cta_with_blocks_of_many_lengths(nb, kind):
         ck.close()
 
 
+@pytest.mark.parametrize("rows", [600, 4_000, 140_000])
+@pytest.mark.parametrize("kind", ["f32", "i32"])
+def test_ties_run_out_on_rows_with_a_short_last_block(rows, kind):
+    """Implicit layout whose rows end in a shorter block (five blocks per row: 8, 8, 8, 8, 5 elements), which the
+    selection treats as a layout of two block lengths; 60 % of the blocks unchanged, k beyond the changed ones, so
+    the ties at zero run out inside one selection CTA and every offset behind depends on which lengths were taken.
+    600 rows: one CTA; 4000 rows: five CTAs of the one-tile kernel; 140 000 rows: several tiles per CTA."""
+    r = rng(77 + rows)
+    row, blk = 37, 8
+    n, nb = rows * row, rows * 5
+    geom = Geometry(n, row, blk, 4)
+    boff = block_offsets(geom)
+    lens = np.diff(boff.astype(np.int64))
+    changed = r.random(nb) < 0.4
+    mask = np.repeat(changed, lens)
+    if kind == "f32":
+        z = r.standard_normal(n).astype(np.float32)
+        x = (z + mask * r.standard_normal(n).astype(np.float32)).astype(np.float32)
+    else:
+        z = r.integers(0, 100, size=n).astype(np.int32)
+        x = (z + mask * r.integers(1, 5, size=n)).astype(np.int32)
+    n_changed = int(changed.sum())
+    for k in (n_changed + nb // 5, n_changed + 1, nb - 1):
+        xd = parity.to_dev(x)
+        ck = parity.make_ctx(xd, z, geom=geom)
+        ora = oracle.priority_save(x, z, boff, k=k)
+        got = parity.check_save(ck, ck.priority_save_k(k), x, z, boff, ora)
+        assert got["exact"], "ties at exactly zero leave no freedom"
+        ck.close()
+
+
 def test_uint64_keys_above_32_bits():
     r = rng(8)
     nb, blk = 4000, 16
