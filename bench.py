@@ -464,6 +464,45 @@ def event_floor(dev, reps=50):
             "what": "a one-element fill between two events, behind a running kernel"}
 
 
+def graph_saves(api, name, dev, reps=20):
+    """The saves of one small parameter set recorded once in a CUDA graph and replayed: what a save costs when
+    its three launches are issued by the device instead of one by one from the host (the sets whose kernels
+    are shorter than a launch call).  Same events, same L2 flush, same reset of the running checkpoint as the
+    eager measurement."""
+    import torch
+
+    geom, z0, x0, r_sweep, _, _ = device_workload(name, 0, 0, dev)
+    s = torch.cuda.Stream()
+    x = x0.clone()
+    torch.cuda.synchronize()
+    ck = api.ScarCheckpoint(x, n_shards=geom.n_shards, row_elems=geom.row_elems, block_elems=geom.block_elems, stream=s)
+    z_lib = ck.views()["z"]
+    flush = L2Flush(dev)
+    out = {}
+    with torch.cuda.stream(s):
+        for r in r_sweep:
+            ck.priority_save(r, sync=False)  # every kernel has run once before anything is recorded
+            s.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                ck.priority_save(r, sync=False)
+            ts = []
+            for _ in range(reps + 3):
+                z_lib.copy_(z0)
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(s)
+                g.replay()
+                b.record(s)
+                b.synchronize()
+                ts.append(a.elapsed_time(b))
+            out[str(r)] = {"save_ms": float(np.median(ts[3:])), "save_ms_min": float(np.min(ts[3:]))}
+            del g
+    s.synchronize()
+    ck.close()
+    return out
+
+
 def summarise(m, peak):
     """Per-r save figures, norm and recovery figures of one measured workload."""
     scanned = 2 * m.n * ELEM
@@ -584,6 +623,8 @@ def run_gpu(args):
                                  gpu_launches=int(mm.launches))
             mm.ck.close()
             del mm
+            torch.cuda.empty_cache()
+            configs[name]["graph_replay"] = graph_saves(api, name, dev)
             torch.cuda.empty_cache()
         line["configs"] = configs
     print(json.dumps(line))
