@@ -84,6 +84,42 @@ template <> struct ScoreKey<unsigned> {  // caller-supplied 32-bit priorities (r
     static __device__ __forceinline__ bool nonfinite(K) { return false; }
 };
 
+// The selection kernels run every instruction once, and their time is close to the number of instructions a warp
+// issues.  Combining the per-warp partials of a CTA-wide sum or scan with a loop over shared memory costs four
+// instructions per warp of the CTA; here every warp takes one partial per lane and combines them with shuffles.
+//
+// Exclusive prefix, for the calling thread's warp, of the NW per-warp partials in sh[]; *total gets their sum.
+template <typename W, int NW>
+__device__ __forceinline__ W warp_partials(const W *sh, W *total) {
+    static_assert(NW <= 32 && (NW & (NW - 1)) == 0, "one partial per lane");
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const W v = lane < NW ? sh[lane] : W(0);
+    W inc = v;
+#pragma unroll
+    for (int o = 1; o < NW; o <<= 1) {
+        const W n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (total) *total = __shfl_sync(0xffffffffu, inc, NW - 1);
+    return __shfl_sync(0xffffffffu, inc - v, w);
+}
+
+// Exclusive prefix sum of one value per thread over a CTA of kSelThreads threads; *total gets the sum.
+template <typename W>
+__device__ __forceinline__ W sel_excl_scan(W v, W *sh /*kSelThreads / 32*/, W *total) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    W inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const W n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    __syncthreads();
+    if (lane == 31) sh[w] = inc;
+    __syncthreads();
+    return warp_partials<W, kSelThreads / 32>(sh, total) + inc - v;
+}
+
 // Sums N values per thread over the CTA with one pair of barriers.  sh holds N * NT / 32 words.
 template <int N, int NT = kThreads>
 __device__ __forceinline__ void cta_sum_n(unsigned long long (&v)[N], unsigned long long *sh) {
@@ -97,12 +133,7 @@ __device__ __forceinline__ void cta_sum_n(unsigned long long (&v)[N], unsigned l
     }
     __syncthreads();
 #pragma unroll
-    for (int i = 0; i < N; ++i) {
-        unsigned long long t = 0;
-#pragma unroll
-        for (int j = 0; j < NT / 32; ++j) t += sh[j * N + i];
-        v[i] = t;
-    }
+    for (int i = 0; i < N; ++i) v[i] = group_sum<32, unsigned long long>(lane < NT / 32 ? sh[lane * N + i] : 0ull);
 }
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned *p) {
@@ -205,7 +236,7 @@ __device__ __forceinline__ unsigned resolve_digit_w(const unsigned *hist, unsign
     unsigned long long sum = 0;
 #pragma unroll
     for (int i = 0; i < per; ++i) sum += local[i];
-    unsigned long long cum = cta_excl_scan<unsigned long long, kSelThreads>(sum, sh_scan, nullptr);
+    unsigned long long cum = sel_excl_scan<unsigned long long>(sum, sh_scan, nullptr);
 #pragma unroll
     for (int i = 0; i < per; ++i) {
         unsigned long long h = local[i];
@@ -289,7 +320,7 @@ __device__ __forceinline__ unsigned long long boundary_len(const S *__restrict__
         for (int j = 0; j < kSelPerThread; ++j)
             if ((valid >> j & 1u) && key[j] == tau) eq_bits |= 1u << j;
         u64 tot;
-        u64 rank = run + cta_excl_scan<u64, kSelThreads>(__popc(eq_bits), sh_scan, &tot);
+        u64 rank = run + sel_excl_scan<u64>(__popc(eq_bits), sh_scan, &tot);
         run += tot;
         for (int j = 0; j < kSelPerThread; ++j)
             if (eq_bits >> j & 1u) {
@@ -424,7 +455,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
         alive = __syncthreads_and(ok) != 0;
         SEL_STAMP(st, 27);  // every CTA's record read
         if (alive) {
-            const u64 ex = cta_excl_scan<u64, kSelThreads>(e, sh_scan, nullptr);
+            const u64 ex = sel_excl_scan<u64>(e, sh_scan, nullptr);
             u64 take = need > ex ? need - ex : 0;
             if (take > e) take = e;
             if (take != 0 && take != e) {  // the tau-keys run out inside CTA c's range
@@ -465,7 +496,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
                     else if (key[j] == tau) eq_bits |= 1u << j;
                 }
             u64 tot_eq;
-            u64 rank = run_eq + cta_excl_scan<u64, kSelThreads>(__popc(eq_bits), sh_scan, &tot_eq);
+            u64 rank = run_eq + sel_excl_scan<u64>(__popc(eq_bits), sh_scan, &tot_eq);
             unsigned take_bits = gt_bits;
             for (int j = 0; j < kSelPerThread; ++j)
                 if (eq_bits >> j & 1u) {
@@ -488,7 +519,7 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
             // lengths below (a buffer has fewer than 2^48 elements: init rejects more)
             u64 tot_both;
             const u64 both =
-                cta_excl_scan<u64, kSelThreads>(((u64)__popc(take_bits) << 48) | lsum, sh_scan, &tot_both);
+                sel_excl_scan<u64>(((u64)__popc(take_bits) << 48) | lsum, sh_scan, &tot_both);
             u64 pos = pos_base + (both >> 48);
             u64 off = off_base + (both & ((1ull << 48) - 1));
 #pragma unroll
@@ -579,13 +610,8 @@ __device__ __forceinline__ bool resolve_digit_when_complete(unsigned *hist, unsi
         if (threadIdx.x == 0)
             sh_stop[iter & 1] = iter > kHistPollLimit || ((iter & 63u) == 63u && ld_acquire(&st->error) != 0);
         __syncthreads();
-        unsigned total = 0, before = 0;
-#pragma unroll
-        for (int i = 0; i < kWarps; ++i) {
-            const unsigned t = buf[i];
-            if (i < w) before += t;
-            total += t;
-        }
+        unsigned total;
+        const unsigned before = warp_partials<unsigned, kWarps>(buf, &total);
         if (total == expected) {
             // exclusive prefix of this thread's bins, highest bins first: warps before, lanes before
             unsigned inc = sum;
@@ -777,15 +803,17 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
             sh_wl[2 * (threadIdx.x >> 5) + 1] = leq;
         }
         __syncthreads();
-        unsigned c_gt = 0, c_eq = 0, t_nf = 0;
+        // one warp's partial per lane (the fields of different warps cannot be added inside one word: up to 4096)
+        const int ln = threadIdx.x & 31;
+        const unsigned pv = ln < kWarps ? sh_w[ln] : 0u;
+        const unsigned c_gt = __reduce_add_sync(0xffffffffu, pv & 1023u);
+        const unsigned c_eq = __reduce_add_sync(0xffffffffu, (pv >> 10) & 1023u);
+        const unsigned t_nf = __reduce_add_sync(0xffffffffu, pv >> 20);
         lgt = leq = 0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            const unsigned v = sh_w[w];
-            c_gt += v & 1023u, c_eq += (v >> 10) & 1023u, t_nf += v >> 20;
+        if (!ulen) {
+            lgt = group_sum<32, u64>(ln < kWarps ? sh_wl[2 * ln] : 0ull);
+            leq = group_sum<32, u64>(ln < kWarps ? sh_wl[2 * ln + 1] : 0ull);
         }
-        if (!ulen)
-            for (int w = 0; w < kWarps; ++w) lgt += sh_wl[2 * w], leq += sh_wl[2 * w + 1];
         my_gt = c_gt, my_eq = c_eq, my_nf = t_nf, my_lgt = lgt, my_leq = leq;
         SEL_STAMP(st, 26);  // own counts known
         if (!SOLO && threadIdx.x == 0) rec_publish(&st->rec[blockIdx.x], c_gt, c_eq, t_nf, lgt, leq);
@@ -812,7 +840,7 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
             // fewer than 2^21 keys in the whole grid (one tile of 4096 per CTA, fewer than 512 CTAs): three
             // 21-bit fields
             u64 tot;
-            const u64 ex = cta_excl_scan<u64, kSelThreads>((u64)gt | ((u64)e << 21) | ((u64)nf << 42), sh_scan64, &tot);
+            const u64 ex = sel_excl_scan<u64>((u64)gt | ((u64)e << 21) | ((u64)nf << 42), sh_scan64, &tot);
             const unsigned ex_gt = (unsigned)(ex & 0x1fffffu), ex_e = (unsigned)((ex >> 21) & 0x1fffffu);
             const unsigned tot_gt = (unsigned)(tot & 0x1fffffu), tot_e = (unsigned)((tot >> 21) & 0x1fffffu);
             total_nf = (unsigned)(tot >> 42);
@@ -865,7 +893,7 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
         if (my_take == my_eq) {
             take_bits |= eq_bits;
         } else if (my_take != 0) {  // only in the CTA where the tau-keys run out (the same decision in all its threads)
-            unsigned rank = cta_excl_scan<unsigned, kSelThreads>(__popc(eq_bits), sh_scan, nullptr);
+            unsigned rank = sel_excl_scan<unsigned>(__popc(eq_bits), sh_scan, nullptr);
             for (int j = 0; j < nv; ++j)
                 if (eq_bits >> j & 1u) {
                     if (rank < my_take) take_bits |= 1u << j;
@@ -873,7 +901,7 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
                 }
         }
         if (ulen) {
-            unsigned pos = my_sel_base + cta_excl_scan<unsigned, kSelThreads>(__popc(take_bits), sh_scan, nullptr);
+            unsigned pos = my_sel_base + sel_excl_scan<unsigned>(__popc(take_bits), sh_scan, nullptr);
             for (int j = 0; j < nv; ++j)
                 if (take_bits >> j & 1u) {
                     sel[pos] = first + j;
@@ -893,7 +921,7 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
             }
             // one scan for both outputs: block counts in the top 16 bits (at most 4096 per tile), summed
             // lengths below (a buffer has fewer than 2^48 elements: init rejects more)
-            const u64 both = cta_excl_scan<u64, kSelThreads>(((u64)__popc(take_bits) << 48) | lsum, sh_scan64, nullptr);
+            const u64 both = sel_excl_scan<u64>(((u64)__popc(take_bits) << 48) | lsum, sh_scan64, nullptr);
             unsigned pos = my_sel_base + (unsigned)(both >> 48);
             u64 off = my_len_base + (both & ((1ull << 48) - 1));
             if (two_len) {
