@@ -675,14 +675,27 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
     const u64 key_or = KT::kSkippable ? st->key_or : ~0ull;  // put back to 0 after the exchange
     const u64 ulen = uniform_block_len(g);
     K *my = sh_key + threadIdx.x * kPad;
+    // 32-bit keys always start with digit pass 0, so its histogram is built here, from the registers the keys were
+    // loaded into: no second walk over them.  (64-bit keys usually skip their first passes.)
+    constexpr bool kFusedFirstPass = !KT::kSkippable;
     int nv;  // how many of this thread's P blocks exist
     {
         K key[P];
         unsigned valid;
-        load_keys<S>(score, B, first, key, valid);
+        load_keys<S>(score, B, first, key, valid);  // on their way while the histogram is cleared
+        for (int i = threadIdx.x; i < kHistBins; i += kSelThreads) sh_hist[i] = 0;
+        if (threadIdx.x == 0) {
+            sh_boundary = -1;
+            sh_boundary_take = 0;
+        }
+        __syncthreads();
         nv = __popc(valid);  // the valid ones come first
 #pragma unroll
-        for (int j = 0; j < P; ++j) my[j] = key[j];
+        for (int j = 0; j < P; ++j) {
+            my[j] = key[j];
+            if (kFusedFirstPass && !none && j < nv)
+                atomicAdd(&sh_hist[(unsigned)((key[j] >> KT::shift(0)) & ((1ull << KT::width(0)) - 1))], 1u);
+        }
     }
     // Rows that end in a shorter block give an implicit layout two block lengths.  Which of this thread's blocks
     // are the short ones is worked out once; every sum of lengths is then two population counts.
@@ -697,11 +710,6 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
             if (j == g.blocks_per_row - 1) short_bits |= 1u << i;
             if (++j == g.blocks_per_row) j = 0;
         }
-    }
-    for (int i = threadIdx.x; i < kHistBins; i += kSelThreads) sh_hist[i] = 0;
-    if (threadIdx.x == 0) {
-        sh_boundary = -1;
-        sh_boundary_take = 0;
     }
     __syncthreads();
     SEL_STAMP(st, 1);  // keys loaded
@@ -722,13 +730,17 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
             // shared histogram, its barrier and the sweep over its bins would cost more.  taking_part is the same
             // number in every CTA, so all of them take the same branch.
             const bool direct = !SOLO && p != 0 && taking_part <= kSelDirectKeys;
+            if (kFusedFirstPass && p == 0) {
+                // counted while the keys were loaded
+            } else {
 #pragma unroll 2
-            for (int j = 0; j < nv; ++j) {
-                const u64 key = my[j];
-                if (p == 0 || (key >> (shift + width)) == prefix) {
-                    const unsigned bin = (unsigned)((key >> shift) & mask);
-                    if (direct) atomicAdd(&st->hist[p][bin], 1u);  // two atomics, not one through a generic pointer
-                    else atomicAdd(&sh_hist[bin], 1u);
+                for (int j = 0; j < nv; ++j) {
+                    const u64 key = my[j];
+                    if (p == 0 || (key >> (shift + width)) == prefix) {
+                        const unsigned bin = (unsigned)((key >> shift) & mask);
+                        if (direct) atomicAdd(&st->hist[p][bin], 1u);
+                        else atomicAdd(&sh_hist[bin], 1u);
+                    }
                 }
             }
             if (!direct) __syncthreads();
