@@ -763,9 +763,9 @@ k_select_tile(const S *__restrict__ score, Geom g, unsigned k, SelState *st, Sav
             unsigned d = 0, h = 0;
             unsigned *hist = SOLO ? sh_hist : st->hist[p];
             const unsigned expected = SOLO ? taking_part : taking_part + never;
-            alive = width == 11
-                        ? resolve_digit_when_complete<11, SOLO>(hist, expected, need, d, h, st, sh_poll, sh_out, sh_stop)
-                        : resolve_digit_when_complete<10, SOLO>(hist, expected, need, d, h, st, sh_poll, sh_out, sh_stop);
+            // one instantiation for both digit widths: a 10-bit pass leaves the upper half of its 2048-bin row at
+            // zero, and code that has already run once is cheaper than a second copy that has not
+            alive = resolve_digit_when_complete<11, SOLO>(hist, expected, need, d, h, st, sh_poll, sh_out, sh_stop);
             if (alive) {
                 prefix = (prefix << width) | d;
                 taking_part = h;  // the keys of the resolved bin are the ones the next pass counts
