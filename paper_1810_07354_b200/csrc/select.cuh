@@ -363,8 +363,12 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
     const unsigned t_hi = t_lo + tiles_per_cta < n_tiles ? t_lo + tiles_per_cta : n_tiles;
     const bool none = k == 0;
     const u64 key_or = KT::kSkippable ? st->key_or : ~0ull;  // put back to 0 after the exchange
-    K key[kSelPerThread];
-    unsigned valid = 0;
+    const u64 ulen = uniform_block_len(g);
+    // Every walk over the CTA's tiles has the next tile's keys on their way while this tile's are worked on: one
+    // CTA per SM keeps few loads in flight otherwise.
+    K key[kSelPerThread], ahead[kSelPerThread];
+    unsigned valid = 0, valid_ahead = 0;
+    const u64 mine0 = (u64)threadIdx.x * kSelPerThread;
     for (int i = threadIdx.x; i < kHistBins; i += kSelThreads) sh_hist[i] = 0;
     if (threadIdx.x == 0) {
         sh_boundary = -1;
@@ -384,8 +388,12 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
                 prefix <<= width;
                 continue;
             }
+            if (t_lo < t_hi) load_keys<S>(score, B, (u64)t_lo * kSelTile + mine0, ahead, valid_ahead);
             for (unsigned t = t_lo; t < t_hi; ++t) {
-                load_keys<S>(score, B, (u64)t * kSelTile + (u64)threadIdx.x * kSelPerThread, key, valid);
+#pragma unroll
+                for (int j = 0; j < kSelPerThread; ++j) key[j] = ahead[j];
+                valid = valid_ahead;
+                if (t + 1 < t_hi) load_keys<S>(score, B, (u64)(t + 1) * kSelTile + mine0, ahead, valid_ahead);
 #pragma unroll
                 for (int j = 0; j < kSelPerThread; ++j) {
                     const bool match = p == 0 || ((u64)key[j] >> (shift + width)) == prefix;
@@ -411,18 +419,23 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
     const K tau = (K)prefix;
 
     // ---- this CTA's record: counts and summed lengths of its keys above / at tau
+    u64 my_eq = 0;
     if (alive) {
         u64 five[5] = {0, 0, 0, 0, 0};  // c_gt, c_eq, c_nf, len_gt, len_eq
+        if (t_lo < t_hi) load_keys<S>(score, B, (u64)t_lo * kSelTile + mine0, ahead, valid_ahead);
         for (unsigned t = t_lo; t < t_hi; ++t) {
-            const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kSelPerThread;
-            load_keys<S>(score, B, first, key, valid);
+            const u64 first = (u64)t * kSelTile + mine0;
+#pragma unroll
+            for (int j = 0; j < kSelPerThread; ++j) key[j] = ahead[j];
+            valid = valid_ahead;
+            if (t + 1 < t_hi) load_keys<S>(score, B, (u64)(t + 1) * kSelTile + mine0, ahead, valid_ahead);
 #pragma unroll
             for (int j = 0; j < kSelPerThread; ++j) {
                 if (!(valid >> j & 1u)) continue;
                 if (SK::nonfinite(key[j])) ++five[2];
                 if (none || key[j] < tau) continue;
-                uint64_t beg, len;
-                g.range((uint32_t)(first + j), beg, len);
+                uint64_t beg, len = 0;
+                if (!ulen) g.range((uint32_t)(first + j), beg, len);  // one block length: lengths are counts
                 if (key[j] > tau) {
                     ++five[0];
                     five[3] += len;
@@ -433,6 +446,8 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
             }
         }
         cta_sum_n<5, kSelThreads>(five, sh_red);
+        if (ulen) five[3] = five[0] * ulen, five[4] = five[1] * ulen;
+        my_eq = five[1];
         SEL_STAMP(st, 26);  // own counts known
         if (threadIdx.x == 0) {
             rec_publish(&st->rec[blockIdx.x], (unsigned)five[0], (unsigned)five[1], (unsigned)five[2], five[3], five[4]);
@@ -484,10 +499,17 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
     SEL_STAMP(st, 28);  // bases known
     // ---- emit: ordered compaction of this CTA's tiles
     if (alive && !none) {
+        // Keys equal to tau: this CTA takes all of its own, none of them, or (one CTA at most) the first few; only
+        // that CTA has to rank them tile by tile.
+        const bool take_none = need <= my_eq_before, take_all = need >= my_eq_before + my_eq;
         u64 run_eq = my_eq_before, pos_base = my_sel_base, off_base = my_len_base;
+        if (t_lo < t_hi) load_keys<S>(score, B, (u64)t_lo * kSelTile + mine0, ahead, valid_ahead);
         for (unsigned t = t_lo; t < t_hi; ++t) {
-            const u64 first = (u64)t * kSelTile + (u64)threadIdx.x * kSelPerThread;
-            load_keys<S>(score, B, first, key, valid);
+            const u64 first = (u64)t * kSelTile + mine0;
+#pragma unroll
+            for (int j = 0; j < kSelPerThread; ++j) key[j] = ahead[j];
+            valid = valid_ahead;
+            if (t + 1 < t_hi) load_keys<S>(score, B, (u64)(t + 1) * kSelTile + mine0, ahead, valid_ahead);
             unsigned gt_bits = 0, eq_bits = 0;
 #pragma unroll
             for (int j = 0; j < kSelPerThread; ++j)
@@ -495,14 +517,32 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
                     if (key[j] > tau) gt_bits |= 1u << j;
                     else if (key[j] == tau) eq_bits |= 1u << j;
                 }
-            u64 tot_eq;
-            u64 rank = run_eq + sel_excl_scan<u64>(__popc(eq_bits), sh_scan, &tot_eq);
             unsigned take_bits = gt_bits;
-            for (int j = 0; j < kSelPerThread; ++j)
-                if (eq_bits >> j & 1u) {
-                    if (rank < need) take_bits |= 1u << j;
-                    ++rank;
-                }
+            if (take_all) {
+                take_bits |= eq_bits;
+            } else if (!take_none) {
+                u64 tot_eq;
+                u64 rank = run_eq + sel_excl_scan<u64>(__popc(eq_bits), sh_scan, &tot_eq);
+                for (int j = 0; j < kSelPerThread; ++j)
+                    if (eq_bits >> j & 1u) {
+                        if (rank < need) take_bits |= 1u << j;
+                        ++rank;
+                    }
+                run_eq += tot_eq;
+            }
+            if (ulen) {  // one block length: an offset is a position times that length
+                u64 tot;
+                u64 pos = pos_base + sel_excl_scan<u64>(__popc(take_bits), sh_scan, &tot);
+#pragma unroll
+                for (int j = 0; j < kSelPerThread; ++j)
+                    if (take_bits >> j & 1u) {
+                        sel[pos] = (uint32_t)(first + j);
+                        poff[pos] = pos * ulen;
+                        ++pos;
+                    }
+                pos_base += tot;
+                continue;
+            }
             u64 lens[kSelPerThread];
             u64 lsum = 0;
 #pragma unroll
@@ -530,7 +570,6 @@ k_select(const S *__restrict__ score, Geom g, unsigned long long k, SelState *st
                     ++pos;
                     off += lens[j];
                 }
-            run_eq += tot_eq;
             pos_base += tot_both >> 48;
             off_base += tot_both & ((1ull << 48) - 1);
         }
