@@ -76,7 +76,7 @@ def oracle_norm(x, z, boff, lost, norm, w):
     return oracle.perturbation_norm_weighted(x, z, boff, lost, norm, w)
 
 
-@pytest.mark.parametrize("seed", range(96))
+@pytest.mark.parametrize("seed", range(256))
 def test_random_case(seed):
     r = rng(1000 + seed)
     layout, boff, x, z, norm, w = random_case(r)
